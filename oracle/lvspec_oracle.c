@@ -1,0 +1,195 @@
+/*
+ * CPU oracle for the LVSpec verify step.  TEST INFRASTRUCTURE ONLY: tests, the
+ * smoke check and the benchmark's CPU-baseline leg may call it; the product
+ * path never does, and it shares no code with the CUDA sources.
+ *
+ * Everything is written out as the plain definition, in fp64, with no tiling,
+ * no online softmax and no reordering, so it can be checked against the paper
+ * by eye.  OpenMP only distributes independent (batch, query, head) units and
+ * independent logits rows over the host cores.
+ *
+ * Pinned by tests/test_oracle_*.py against: torch's scaled-dot-product
+ * attention in fp64 (the attention the paper names in App. "Baseline
+ * Details"), closed forms (identical keys, dominant key, key translation),
+ * brute-force enumeration and hand-worked cases of the rule (tests/golden),
+ * and the closed form of Prop. 2.2.  The paper prints no worked numeric
+ * example of the rule, so beyond those pins the rule is "parity unpinned"
+ * against the authors' own code.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+static double bf16_to_double(uint16_t bits)
+{
+    uint32_t u = ((uint32_t)bits) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/*
+ * Verification attention of the gamma draft queries over the cache (Eq. 1: the
+ * target model verifies the K draft tokens in one parallel pass; the attention
+ * is scaled-dot-product attention, App. "Baseline Details"), plus the visual
+ * mass: the share of each query's softmax that lands on the visual span.
+ *
+ *   q         bf16 bits [B, gamma, Hq, D]
+ *   k, v      bf16 bits [B, Hkv, Lmax, D]
+ *   kv_len    [B]   cache length including the gamma draft slots (the last ones)
+ *   span      [B,2] visual positions [start, end)
+ *   out       fp64 [B, gamma, Hq, D]
+ *   mass      fp64 [B, gamma, Hq]
+ *   probs     optional fp64 [B, gamma, Hq, Lmax] (0 beyond the visible prefix)
+ *
+ * Query g of a sequence sees positions j < kv_len - gamma + g + 1 (causal over
+ * the draft tail).  Head h reads KV head h / (Hq / Hkv).
+ */
+void lvspec_oracle_verify_attention(const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                                    const int32_t *kv_len, const int32_t *span,
+                                    int B, int gamma, int Hq, int Hkv, int D, int Lmax,
+                                    double *out, double *mass, double *probs)
+{
+    const int G = Hq / Hkv;
+    const double scale = 1.0 / sqrt((double)D);
+    const long units = (long)B * gamma * Hq;
+#pragma omp parallel
+    {
+        double *s = (double *)malloc(sizeof(double) * (size_t)(Lmax > 0 ? Lmax : 1));
+        double *qd = (double *)malloc(sizeof(double) * (size_t)D);
+#pragma omp for schedule(dynamic, 1)
+        for (long u = 0; u < units; ++u) {
+            const int h = (int)(u % Hq);
+            const int g = (int)((u / Hq) % gamma);
+            const int b = (int)(u / ((long)Hq * gamma));
+            const int kvh = h / G;
+            const int vis = kv_len[b] - gamma + g + 1;
+            const int vs = span[2 * b], ve = span[2 * b + 1];
+            const uint16_t *qrow = q + (((size_t)b * gamma + g) * Hq + h) * D;
+            const uint16_t *kb = k + ((size_t)b * Hkv + kvh) * (size_t)Lmax * D;
+            const uint16_t *vb = v + ((size_t)b * Hkv + kvh) * (size_t)Lmax * D;
+            double *orow = out + (((size_t)b * gamma + g) * Hq + h) * D;
+
+            for (int d = 0; d < D; ++d) qd[d] = bf16_to_double(qrow[d]);
+            double m = -INFINITY;
+            for (int j = 0; j < vis; ++j) {
+                double acc = 0.0;
+                for (int d = 0; d < D; ++d) acc += qd[d] * bf16_to_double(kb[(size_t)j * D + d]);
+                s[j] = acc * scale;
+                if (s[j] > m) m = s[j];
+            }
+            double Z = 0.0;
+            for (int j = 0; j < vis; ++j) { s[j] = exp(s[j] - m); Z += s[j]; }
+            for (int d = 0; d < D; ++d) orow[d] = 0.0;
+            double vm = 0.0;
+            for (int j = 0; j < vis; ++j) {
+                const double p = s[j] / Z;
+                if (j >= vs && j < ve) vm += p;
+                for (int d = 0; d < D; ++d) orow[d] += p * bf16_to_double(vb[(size_t)j * D + d]);
+                if (probs) probs[(((size_t)b * gamma + g) * Hq + h) * (size_t)Lmax + j] = p;
+            }
+            if (probs)
+                for (int j = vis > 0 ? vis : 0; j < Lmax; ++j)
+                    probs[(((size_t)b * gamma + g) * Hq + h) * (size_t)Lmax + j] = 0.0;
+            mass[((size_t)b * gamma + g) * Hq + h] = vm;
+        }
+        free(s);
+        free(qd);
+    }
+}
+
+/* Ordering used for the loosened set: score ascending, then position ascending
+ * (a stable ascending argsort). */
+typedef struct { double score; int pos; } scored_t;
+static int cmp_scored(const void *a, const void *b)
+{
+    const scored_t *x = (const scored_t *)a, *y = (const scored_t *)b;
+    if (x->score < y->score) return -1;
+    if (x->score > y->score) return 1;
+    return (x->pos > y->pos) - (x->pos < y->pos);
+}
+
+/*
+ * Loose acceptance pass (Sec. 3.2 and 3.3).
+ *
+ *   logits   fp32 [B, gamma, V]   target logits, row i judges draft token i
+ *   draft    int32 [B, gamma]
+ *   mass     fp32 [B, gamma, Hm]  per-head relevance; Hm = 1 takes a ready score
+ *   n_loose  number of loosened positions (the "lambda K lowest" of Eq. 5)
+ *   window   shift tolerance W: 0 switches PST off, W >= gamma - 1 is Eq. 7
+ *   accept_len int32 [B]; target int32 [B,gamma] and acc uint8 [B,gamma] optional
+ *
+ * Steps, in the paper's order:
+ *  1. y_i = the target's token at position i: the largest logit, first
+ *     occurrence on ties; NaN counts as -inf; a row with nothing above -inf
+ *     gives token 0.
+ *  2. score_i = sum over heads of mass (added in index order, in double).
+ *  3. I' = the first n_loose positions of the ascending stable argsort (Eq. 5).
+ *  4. nabla_i = 1 if draft_i == y_i; else 1 if i in I'; else 1 if y_i equals a
+ *     draft token at a position within W of i; else 0 (Eq. 6 / Eq. 7).
+ *  5. accepted length = sum_k prod_{j<=k} nabla_j (Eq. 2).
+ */
+void lvspec_oracle_loose_accept(const float *logits, const int32_t *draft, const float *mass,
+                                int B, int gamma, int V, int Hm, int n_loose, int window,
+                                int32_t *accept_len, int32_t *target, uint8_t *acc)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        int32_t *y = (int32_t *)malloc(sizeof(int32_t) * (size_t)(gamma > 0 ? gamma : 1));
+        uint8_t *nabla = (uint8_t *)malloc((size_t)(gamma > 0 ? gamma : 1));
+        uint8_t *loosened = (uint8_t *)calloc((size_t)(gamma > 0 ? gamma : 1), 1);
+        scored_t *order = (scored_t *)malloc(sizeof(scored_t) * (size_t)(gamma > 0 ? gamma : 1));
+
+        for (int i = 0; i < gamma; ++i) {
+            const float *row = logits + ((size_t)b * gamma + i) * (size_t)V;
+            float best = -INFINITY;
+            int arg = 0;
+            for (int t = 0; t < V; ++t) {
+                const float x = row[t];
+                if (x > best) { best = x; arg = t; }   /* NaN never wins; first max kept */
+            }
+            y[i] = arg;
+        }
+        for (int i = 0; i < gamma; ++i) {
+            double sc = 0.0;
+            for (int h = 0; h < Hm; ++h) sc += (double)mass[((size_t)b * gamma + i) * Hm + h];
+            order[i].score = sc;
+            order[i].pos = i;
+        }
+        qsort(order, (size_t)gamma, sizeof(scored_t), cmp_scored);
+        for (int r = 0; r < gamma && r < n_loose; ++r) loosened[order[r].pos] = 1;
+
+        for (int i = 0; i < gamma; ++i) {
+            const int32_t *dr = draft + (size_t)b * gamma;
+            int ok = (dr[i] == y[i]);
+            if (!ok && loosened[i]) ok = 1;
+            if (!ok) {
+                for (int kk = 0; kk < gamma; ++kk) {
+                    const int dist = kk > i ? kk - i : i - kk;
+                    if (dist <= window && dr[kk] == y[i]) { ok = 1; break; }
+                }
+            }
+            nabla[i] = (uint8_t)ok;
+        }
+        int tau = 0;
+        for (int kk = 0; kk < gamma; ++kk) {
+            int prod = 1;
+            for (int j = 0; j <= kk; ++j) prod *= nabla[j];
+            tau += prod;
+        }
+        accept_len[b] = tau;
+        if (target) memcpy(target + (size_t)b * gamma, y, sizeof(int32_t) * (size_t)gamma);
+        if (acc) memcpy(acc + (size_t)b * gamma, nabla, (size_t)gamma);
+        free(y); free(nabla); free(loosened); free(order);
+    }
+}
+
+/* Number of loosened positions for a loose parameter lambda (Sec. 3.2: "the
+ * lambda K tokens with the lowest scores"; the slice 0:lambda K of Eq. 5).  A
+ * non-integer product is cut down to the integer below; 1e-9 guards products
+ * that land a rounding error under an integer. */
+int lvspec_oracle_n_loose(double lambda, int gamma)
+{
+    return (int)floor(lambda * (double)gamma + 1e-9);
+}
