@@ -1,0 +1,404 @@
+"""Benchmark of the LVSpec verify step on B200.
+
+A "step" is one pass of the whole hot path over one batch of synthetic input:
+the verification attention of every layer of the model-shaped config (each
+layer with its own K/V cache), then the loose acceptance pass over the target
+logits fed by the last layer's visual mass.
+
+    python bench.py --gpus N --steps K --warmup W [--config ID] [--impl reference]
+
+prints one JSON line.  The path does not shard ("replicas only"): with N > 1
+every rank runs the same workload on its own GPU, no collective on the data
+path; the value is the sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "verified draft tokens/sec per verify step"
+UNIT = "tokens/s"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="BASELINE config id (1, 2 or 3)")
+    ap.add_argument("--kernel", type=int, default=0, help="attention kernel selector (0 = default)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch layer by layer, no CUDA graph")
+    return ap.parse_args()
+
+
+# --------------------------------------------------------------------------- #
+# clocks
+# --------------------------------------------------------------------------- #
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed
+    region runs (reads settings only)."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self._stop = threading.Event()
+        self._thread = None
+
+    def _once(self):
+        try:
+            out = subprocess.run(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                  "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
+            parts = [x.strip() for x in out.strip().split(",")]
+            if len(parts) >= 6:
+                self.samples.append(parts)
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self._stop.is_set():
+            self._once()
+            self._stop.wait(0.1)
+
+    def start(self):
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join(timeout=10)
+        if not self.samples:
+            self._once()
+
+    def summary(self):
+        sm = [float(s[0]) for s in self.samples if s[0].replace(".", "").isdigit()]
+        mx = [float(s[1]) for s in self.samples if s[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(s[2 + i].lower() == "active" for s in self.samples)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------- #
+# reference arm: the CPU oracle, as it stands, on a bounded sample
+# --------------------------------------------------------------------------- #
+def oracle_sample_step(cfg, sample_layers: int):
+    """Times the oracle on `sample_layers` layers of attention plus the
+    acceptance pass and scales the attention part to the config's layer count.
+    Returns (seconds per full step, cores used)."""
+    import oracle
+    from paper_2604_05650_b200 import workloads as W
+    cores = oracle.max_threads()
+    t_attn = 0.0
+    mass = None
+    for layer in range(sample_layers):
+        q, k, v, kv_len, span = W.attention_inputs(cfg, layer=layer)
+        t0 = time.perf_counter()
+        _, mass = oracle.verify_attention(q, k, v, kv_len, span)
+        t_attn += time.perf_counter() - t0
+    logits, draft = W.accept_inputs(cfg)
+    t0 = time.perf_counter()
+    oracle.loose_accept(logits, draft, mass.astype(np.float32), oracle.n_loose(cfg.lam, cfg.gamma),
+                        cfg.shift_window)
+    t_acc = time.perf_counter() - t0
+    return t_attn * cfg.layers / sample_layers + t_acc, cores
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample_layers = 2
+    for _ in range(max(1, min(args.warmup, 1))):
+        oracle_sample_step(cfg, 1)
+    times = []
+    cores = 1
+    for _ in range(max(1, args.steps)):
+        t, cores = oracle_sample_step(cfg, sample_layers)
+        times.append(t)
+    t_step = sum(times) / len(times)
+    value = cfg.batch * cfg.gamma / t_step
+    sample = (f"each step: {sample_layers} of {cfg.layers} attention layers timed and scaled by layer count, "
+              f"plus the full acceptance pass")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_step * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": workload_desc(cfg, args.gpus),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def workload_desc(cfg, n_gpus):
+    return {"workload": f"BASELINE config {cfg_id_of(cfg)}: {cfg.name}-shaped verify step, {cfg.layers} layers, "
+                        f"batch {cfg.batch}, gamma {cfg.gamma}, heads {cfg.n_q_heads}/{cfg.n_kv_heads}x{cfg.head_dim}, "
+                        f"KV {cfg.kv_len} ({cfg.span[1] - cfg.span[0]} visual), vocab {cfg.vocab}",
+            "kv_bytes_per_step": cfg.kv_bytes_per_layer * cfg.layers,
+            "l2": "inputs larger than L2 (every layer streams its own K/V cache)",
+            "parallelism": "replicas only" if n_gpus > 1 else "1 GPU"}
+
+
+def cfg_id_of(cfg):
+    from paper_2604_05650_b200 import workloads as W
+    for i, c in W.CONFIGS.items():
+        if c is cfg:
+            return i
+    return -1
+
+
+# --------------------------------------------------------------------------- #
+# our arm
+# --------------------------------------------------------------------------- #
+def device_workload(cfg, dev, torch):
+    """Synthetic inputs of the config's recipe drawn on the device (seeded):
+    Q, K, V ~ N(0,1) in bf16 with the +0.5 shift of visual keys on 8 coordinates
+    per KV head; logits and drafts come from the shared host generator."""
+    from paper_2604_05650_b200 import workloads as W
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(cfg.seed)
+    B, g, Hq, Hkv, D, L = cfg.batch, cfg.gamma, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.kv_len
+    vs, ve = cfg.span
+    qs, ks, vs_ = [], [], []
+    for _ in range(cfg.layers):
+        q = torch.randn((B, g, Hq, D), generator=gen, device=dev, dtype=torch.float32)
+        k = torch.randn((B, Hkv, L, D), generator=gen, device=dev, dtype=torch.float32)
+        v = torch.randn((B, Hkv, L, D), generator=gen, device=dev, dtype=torch.float32)
+        for h in range(Hkv):
+            dims = torch.randperm(D, generator=gen, device=dev)[:8]
+            k[:, h, vs:ve, dims] += 0.5
+        qs.append(q.to(torch.bfloat16))
+        ks.append(k.to(torch.bfloat16))
+        vs_.append(v.to(torch.bfloat16))
+        del q, k, v
+    logits, draft = W.accept_inputs(cfg)
+    return qs, ks, vs_, torch.from_numpy(logits).to(dev), torch.from_numpy(draft).to(dev)
+
+
+def run_ours(args, cfg):
+    import torch
+    import torch.distributed as dist
+    from paper_2604_05650_b200 import binding, build as _build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    ctx = binding.Context(local)
+    stream = torch.cuda.Stream(device=dev)
+    ctx.set_stream(stream.cuda_stream)
+    qs, ks, vs_, logits, draft = device_workload(cfg, dev, torch)
+    B, g, Hq, Hkv, D, L = cfg.batch, cfg.gamma, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.kv_len
+    shape = binding.attn_shape(B, g, Hq, Hkv, D, L, 0, args.kernel)
+    kv_len = np.full((B,), L, dtype=np.int32)
+    span = np.tile(np.asarray([cfg.span], dtype=np.int32), (B, 1))
+    out = torch.empty((B, g, Hq, D), dtype=torch.bfloat16, device=dev)
+    mass = torch.empty((B, g, Hq), dtype=torch.float32, device=dev)
+    alen = torch.zeros((B,), dtype=torch.int32, device=dev)
+    torch.cuda.synchronize(dev)
+
+    def attention_layers():
+        for l in range(cfg.layers):
+            ctx.verify_attention(shape, qs[l], ks[l], vs_[l], kv_len, span, out, mass)
+
+    def accept():
+        ctx.loose_accept(B, g, cfg.vocab, Hq, logits, draft, mass, alen, cfg.shift_window, lam=cfg.lam)
+
+    # one warm, un-captured step sizes the scratch memory before any capture
+    with torch.cuda.stream(stream):
+        attention_layers()
+        accept()
+    stream.synchronize()
+    l0 = ctx.launch_count()
+    with torch.cuda.stream(stream):
+        attention_layers()
+        accept()
+    stream.synchronize()
+    launches_per_step = ctx.launch_count() - l0
+
+    graph_attn = graph_acc = None
+    if not args.no_graph:
+        graph_attn, graph_acc = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph_attn, stream=stream):
+            attention_layers()
+        with torch.cuda.graph(graph_acc, stream=stream):
+            accept()
+
+    def step(ev_a=None, ev_b=None):
+        """One verify step on `stream`; ev_a/ev_b bracket the attention part."""
+        if ev_a is not None:
+            ev_a.record(stream)
+        if graph_attn is not None:
+            graph_attn.replay()
+        else:
+            attention_layers()
+        if ev_b is not None:
+            ev_b.record(stream)
+        if graph_acc is not None:
+            graph_acc.replay()
+        else:
+            accept()
+
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3)):
+            step()
+    stream.synchronize()
+
+    clocks = ClockSampler(local)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    attn_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(args.steps)]
+    barrier()
+    torch.cuda.synchronize(dev)
+    clocks.start()
+    with torch.cuda.stream(stream):
+        ev0.record(stream)
+        for i in range(args.steps):
+            step(*attn_ev[i])
+        ev1.record(stream)
+    stream.synchronize()
+    torch.cuda.synchronize(dev)
+    barrier()
+    clocks.stop()
+    status = ctx.device_status()
+    ms_total = ev0.elapsed_time(ev1)
+    ms_attn = sum(a.elapsed_time(b) for a, b in attn_ev) / args.steps
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total_max = float(t.item())
+    ms_step = ms_total_max / args.steps
+    value = world * B * g / (ms_step * 1e-3)
+    accepted = int(alen.sum().item())
+
+    # roofline of the dominant kernel: one verification-attention launch
+    bytes_per_launch = cfg.kv_bytes_per_layer + 2 * (B * g * Hq * D * 2) + B * g * Hq * 4
+    us_per_launch = ms_attn * 1e3 / cfg.layers
+    achieved = bytes_per_launch / (us_per_launch * 1e-6) / 1e9
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    else:
+        peak, peak_src = 6650.0, "fallback"
+    traffic = None
+    tr_path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tr_path):
+        traffic = json.load(open(tr_path)).get(f"config{cfg_id_of(cfg)}")
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": traffic, "peak_source": peak_src, "kernel": "verify attention (one layer)",
+                "us_per_launch": us_per_launch, "bytes_per_launch": bytes_per_launch,
+                "frac_of_nominal_8000": achieved / 8000.0}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": workload_desc(cfg, world), "accepted_tokens_per_s": world * accepted / (ms_step * 1e-3),
+            "accept_len": accepted, "ms_attention_per_step": ms_attn,
+            "ms_accept_per_step": ms_step - ms_attn if world == 1 else None,
+            "gpu_launches": launches_per_step * args.steps, "device_status": status,
+            "cuda_graph": graph_attn is not None, "roofline": roofline, "clocks": clocks.summary()}
+
+    # end to end through the host-buffer entry points
+    if not args.no_e2e:
+        line["e2e"] = run_e2e(args, cfg, ctx, stream, qs, ks, vs_, logits, draft, torch, dev, world, barrier, dist)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        t_cpu, cores = oracle_sample_step(cfg, 8 if cfg.layers >= 8 else cfg.layers)
+        line["cpu_baseline"] = {"value": B * g / t_cpu, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"{min(8, cfg.layers)} of {cfg.layers} attention layers timed once and scaled "
+                                          f"by layer count, plus the full acceptance pass"}
+    ctx.close()
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, cfg, ctx, stream, qs, ks, vs_, logits, draft, torch, dev, world, barrier, dist):
+    """Same step through lvspec_*_host: every input starts in pinned host
+    memory (K/V caches included) and the accepted length ends on the host."""
+    from paper_2604_05650_b200 import binding
+    B, g, Hq, Hkv, D, L = cfg.batch, cfg.gamma, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.kv_len
+    pin = lambda t: t.cpu().pin_memory()
+    hq = [pin(t) for t in qs]
+    hk = [pin(t) for t in ks]
+    hv = [pin(t) for t in vs_]
+    hlog, hdraft = pin(logits), pin(draft)
+    hout = torch.empty((B, g, Hq, D), dtype=torch.bfloat16).pin_memory()
+    hmass = torch.empty((B, g, Hq), dtype=torch.float32).pin_memory()
+    hlen = torch.zeros((B,), dtype=torch.int32).pin_memory()
+    shape = binding.attn_shape(B, g, Hq, Hkv, D, L, 0, args.kernel)
+    kv_len = np.full((B,), L, dtype=np.int32)
+    span = np.tile(np.asarray([cfg.span], dtype=np.int32), (B, 1))
+
+    def step():
+        for l in range(cfg.layers):
+            ctx.verify_attention_host(shape, hq[l], hk[l], hv[l], kv_len, span, hout, hmass)
+        ctx.loose_accept_host(B, g, cfg.vocab, Hq, hlog, hdraft, hmass, hlen, cfg.shift_window, lam=cfg.lam)
+
+    steps = max(1, min(args.steps, 3))
+    step()
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    ev0.record(stream)
+    for _ in range(steps):
+        step()
+    ev1.record(stream)
+    stream.synchronize()
+    barrier()
+    ms = ev0.elapsed_time(ev1) / steps
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = float(t.item())
+    h2d = cfg.layers * (hq[0].numel() * 2 + 2 * hk[0].numel() * 2) + hlog.numel() * 4 + hdraft.numel() * 4 \
+        + hmass.numel() * 4
+    d2h = cfg.layers * (hout.numel() * 2 + hmass.numel() * 4) + hlen.numel() * 4
+    return {"value": world * B * g / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": ms, "steps": steps,
+            "note": "K/V caches of every layer cross PCIe each step"}
+
+
+def main():
+    args = parse()
+    from paper_2604_05650_b200 import workloads as W
+    cfg = W.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,226 @@
+/*
+ * lvspec.h - C ABI of the B200 (sm_100a) hot path of the LVSpec verify step.
+ *
+ * Two operations, in the order a verify step runs them:
+ *
+ *   lvspec_verify_attention  the target model's verification attention: the
+ *       gamma (= the paper's K, Eq. 1) draft-token queries of each sequence
+ *       attend over that sequence's KV cache, which video tokens dominate;
+ *       fused into the softmax is the share of each query's probability that
+ *       lands on the visual-token span ("visual mass"), the relevance score
+ *       this library feeds to the acceptance rule.
+ *
+ *   lvspec_loose_accept      the loose acceptance pass over the target logits:
+ *       vocabulary-wide argmax per draft position, then the rule of Sec. 3.2
+ *       and 3.3 (Eq. 5-7) and the accepted length of Eq. 2.
+ *
+ * Conventions
+ *   - "device" pointers are CUDA global memory of the context's device; "host"
+ *     pointers are ordinary host memory.  The caller owns every buffer it
+ *     passes; the library neither frees nor keeps them past the call.
+ *   - All tensors are dense, row-major, innermost dimension contiguous, with the
+ *     shapes given at each call; device tensors must be 16-byte aligned.
+ *   - Device calls enqueue work on the context's stream and return without
+ *     synchronising.  The return value reports argument and launch errors only.
+ *     A call that returns anything but LVSPEC_OK has launched nothing.
+ *   - A context owns scratch memory on its device and is not thread-safe.
+ *     Calls on one context must not overlap on the GPU with each other unless
+ *     they are ordered on the same stream.
+ *   - There is no CPU fallback: without a CUDA device lvspec_create fails.
+ */
+#ifndef LVSPEC_H_
+#define LVSPEC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LVSPEC_OK = 0,
+    LVSPEC_ERR_INVALID_ARG = 1,  /* null pointer, bad shape, span or length out of range */
+    LVSPEC_ERR_UNSUPPORTED = 2,  /* a shape the kernels do not cover (see each call) */
+    LVSPEC_ERR_WORKSPACE = 3,    /* scratch memory could not be allocated */
+    LVSPEC_ERR_CUDA = 4,         /* a CUDA runtime call failed; see lvspec_last_error */
+    LVSPEC_ERR_TIMEOUT = 5       /* a bounded device-side wait ran out */
+} lvspec_status_t;
+
+/* Bits of the device status word (lvspec_device_status). */
+#define LVSPEC_DEV_WAIT_EXPIRED 0x1u /* a bounded barrier wait gave up; results invalid */
+#define LVSPEC_DEV_NAN_LOGIT    0x2u /* a NaN logit was seen (it was ranked as -inf) */
+
+#define LVSPEC_MAX_BATCH 128   /* sequences per call */
+#define LVSPEC_MAX_ROWS  128   /* gamma * (Hq / Hkv): query rows sharing one KV head */
+#define LVSPEC_MAX_GAMMA 64    /* draft tokens per sequence */
+
+typedef struct lvspec_ctx lvspec_ctx_t; /* opaque */
+
+/* Shape of one verification-attention call. */
+typedef struct {
+    int32_t batch;       /* B, 1..LVSPEC_MAX_BATCH */
+    int32_t gamma;       /* draft queries per sequence, 1..LVSPEC_MAX_GAMMA */
+    int32_t n_q_heads;   /* Hq */
+    int32_t n_kv_heads;  /* Hkv, divides Hq; gamma * Hq / Hkv <= LVSPEC_MAX_ROWS */
+    int32_t head_dim;    /* D: 64 or 128 */
+    int32_t kv_capacity; /* Lmax: cache slots allocated per (sequence, KV head) */
+    int32_t n_split;     /* KV splits per (sequence, KV head); 0 lets the library choose */
+    int32_t kernel;      /* LVSPEC_KERNEL_* ; 0 = default */
+} lvspec_attn_shape_t;
+
+#define LVSPEC_KERNEL_DEFAULT 0
+#define LVSPEC_KERNEL_SIMT    1 /* plain CUDA-core kernel: any supported shape */
+#define LVSPEC_KERNEL_TCGEN05 2 /* TMA + tcgen05 tensor-core kernel */
+
+/* Parameters of the rule.  n_loose >= 0 gives the number of loosened positions
+ * directly; n_loose < 0 derives it from lambda as floor(lambda * gamma + 1e-9)
+ * (Sec. 3.2: the lambda*K positions of lowest relevance; the paper runs
+ * lambda = 0.7, K = 10, i.e. 7 loosened positions). */
+typedef struct {
+    double lambda;   /* in [0, 1]; used when n_loose < 0 */
+    int32_t n_loose; /* -1, or 0..gamma */
+    int32_t reserved;
+} lvspec_thresholds_t;
+
+/* ---- context -------------------------------------------------------------- */
+
+/* Creates a context on CUDA device `device` (it becomes the current device of
+ * the calling thread during each call).  Allocates the scratch memory the
+ * kernels need (a few MiB, grown on demand by later calls) and zeroes it.
+ * Errors: INVALID_ARG (null out pointer, bad ordinal), CUDA (no device or
+ * driver), WORKSPACE. */
+lvspec_status_t lvspec_create(lvspec_ctx_t **ctx, int device);
+
+/* Synchronises the context's stream, frees its scratch memory and the context. */
+lvspec_status_t lvspec_destroy(lvspec_ctx_t *ctx);
+
+/* Sets the CUDA stream (a cudaStream_t passed as void*; NULL = default stream)
+ * that later calls enqueue on. */
+lvspec_status_t lvspec_set_stream(lvspec_ctx_t *ctx, void *cuda_stream);
+
+/* Synchronises the stream, reads and clears the device status word.
+ * `flags` (host) receives the LVSPEC_DEV_* bits.  Returns LVSPEC_ERR_TIMEOUT if
+ * LVSPEC_DEV_WAIT_EXPIRED is set, LVSPEC_ERR_CUDA if the sync failed. */
+lvspec_status_t lvspec_device_status(lvspec_ctx_t *ctx, uint32_t *flags);
+
+/* Text of the last error recorded on this context (never NULL; valid until the
+ * next call on the context).  `ctx` may be NULL: then the text describes why
+ * the last lvspec_create on this thread failed. */
+const char *lvspec_last_error(const lvspec_ctx_t *ctx);
+
+const char *lvspec_status_string(lvspec_status_t status);
+
+/* Number of kernels this context has launched since it was created. */
+uint64_t lvspec_launch_count(const lvspec_ctx_t *ctx);
+
+/* KV splits the library would use for `shape` with the longest sequence
+ * `max_kv_len` (what n_split = 0 resolves to); 0 on invalid input. */
+int32_t lvspec_attention_splits(const lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                int32_t max_kv_len);
+
+/* ---- verification attention ---------------------------------------------------
+ *
+ * Operation (Eq. 1: the K draft tokens are verified by the target model in one
+ * parallel pass; the attention is scaled-dot-product attention, App. "Baseline
+ * Details").  For sequence b, draft query g in [0, gamma), query head h:
+ *
+ *   visible(b, g) = kv_len[b] - gamma + g + 1      (the draft tokens occupy the
+ *                   last gamma slots of the cache and see each other causally)
+ *   s_j   = <q[b,g,h,:], k_cache[b, h / (Hq/Hkv), j, :]> / sqrt(D),  j < visible
+ *   p_j   = softmax_j(s_j)
+ *   out[b,g,h,:]        = sum_j p_j * v_cache[b, h / (Hq/Hkv), j, :]
+ *   visual_mass[b,g,h]  = sum of p_j over j in [span_start, span_end), j < visible
+ *
+ *   q            device, bf16  [B, gamma, Hq, D]
+ *   k_cache      device, bf16  [B, Hkv, Lmax, D]
+ *   v_cache      device, bf16  [B, Hkv, Lmax, D]
+ *   kv_len       host,  int32  [B]      gamma <= kv_len[b] <= Lmax, counts the draft slots
+ *   visual_span  host,  int32  [B][2]   0 <= start <= end <= kv_len[b] - gamma
+ *   out          device, bf16  [B, gamma, Hq, D]   (written)
+ *   visual_mass  device, fp32  [B, gamma, Hq]      (written)
+ *
+ * Products are bf16 x bf16 accumulated in fp32; the softmax, its sums and the
+ * visual mass are fp32; `out` is rounded to bf16 once at the end.  kv_len and
+ * visual_span are read during the call and may be reused as soon as it returns.
+ *
+ * Errors: INVALID_ARG for null pointers, misaligned device pointers, Hq not a
+ * multiple of Hkv, lengths or spans outside the ranges above, batch or gamma
+ * beyond the LVSPEC_MAX_* limits; UNSUPPORTED for head_dim other than 64 / 128
+ * or more than LVSPEC_MAX_ROWS query rows per KV head; WORKSPACE / CUDA.
+ */
+lvspec_status_t lvspec_verify_attention(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                        const void *q, const void *k_cache, const void *v_cache,
+                                        const int32_t *kv_len, const int32_t *visual_span,
+                                        void *out, float *visual_mass);
+
+/* Same operation on HOST buffers: copies q, the caches, and the results through
+ * device staging memory the context owns (grown on demand), on the context's
+ * stream, and synchronises before returning.  All seven arrays are host
+ * pointers with the shapes above (out is bf16, visual_mass fp32). */
+lvspec_status_t lvspec_verify_attention_host(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                             const void *q, const void *k_cache,
+                                             const void *v_cache, const int32_t *kv_len,
+                                             const int32_t *visual_span, void *out,
+                                             float *visual_mass);
+
+/* ---- loose acceptance ---------------------------------------------------------
+ *
+ * Operation, per sequence b (Sec. 3.2, 3.3):
+ *   1. y_i = argmax_v target_logits[b,i,v]; ties go to the lowest v; a NaN
+ *      logit ranks as -inf (and raises LVSPEC_DEV_NAN_LOGIT); a row with
+ *      nothing above -inf gives y_i = 0.
+ *   2. score_i = sum_h visual_mass[b,i,h], added in index order in fp64.
+ *      n_mass_heads = 1 takes a ready per-position score instead (for
+ *      instance the paper's own relevance score of Eq. 4).
+ *   3. Loosened set I' = the first n' positions when positions are ordered by
+ *      (score ascending, position ascending) (Eq. 5).  NaN scores are not
+ *      supported.
+ *   4. accepted_i = (draft_i == y_i) or (i in I') or (y_i == draft_k for some k
+ *      with |k - i| <= shift_window, 0 <= k < gamma)  (Eq. 6; Eq. 7 when
+ *      shift_window >= gamma - 1; shift_window = 0 switches the
+ *      position-shift tolerance off).
+ *   5. accept_len[b] = number of leading accepted positions (Eq. 2), 0..gamma.
+ *
+ *   target_logits  device, fp32  [B, gamma, V]
+ *   draft_tokens   device, int32 [B, gamma]
+ *   visual_mass    device, fp32  [B, gamma, n_mass_heads]
+ *   thresholds     host
+ *   accept_len     device, int32 [B]            (written)
+ *
+ * All decisions are exact integer / IEEE comparisons: the result is
+ * bit-identical to the definition above.
+ * Errors: INVALID_ARG (null or misaligned pointers, batch/gamma/vocab/heads
+ * < 1 or beyond limits, lambda outside [0,1], n_loose > gamma, shift_window
+ * < 0); WORKSPACE / CUDA.
+ */
+lvspec_status_t lvspec_loose_accept(lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,
+                                    int32_t vocab, int32_t n_mass_heads,
+                                    const float *target_logits, const int32_t *draft_tokens,
+                                    const float *visual_mass,
+                                    const lvspec_thresholds_t *thresholds, int32_t shift_window,
+                                    int32_t *accept_len);
+
+/* As lvspec_loose_accept, with two optional extra outputs (either may be NULL):
+ *   target_tokens  device, int32 [B, gamma]   y_i of step 1
+ *   accepted       device, uint8 [B, gamma]   accepted_i of step 4 */
+lvspec_status_t lvspec_loose_accept_ex(lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,
+                                       int32_t vocab, int32_t n_mass_heads,
+                                       const float *target_logits, const int32_t *draft_tokens,
+                                       const float *visual_mass,
+                                       const lvspec_thresholds_t *thresholds,
+                                       int32_t shift_window, int32_t *accept_len,
+                                       int32_t *target_tokens, uint8_t *accepted);
+
+/* Same operation on HOST buffers (see lvspec_verify_attention_host). */
+lvspec_status_t lvspec_loose_accept_host(lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,
+                                         int32_t vocab, int32_t n_mass_heads,
+                                         const float *target_logits, const int32_t *draft_tokens,
+                                         const float *visual_mass,
+                                         const lvspec_thresholds_t *thresholds,
+                                         int32_t shift_window, int32_t *accept_len);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LVSPEC_H_ */

@@ -1,0 +1,200 @@
+"""Thin ctypes binding of liblvspec.so: argument marshalling only.
+
+Every step of the verify path runs in the library's CUDA kernels.  There is no
+CPU fallback: if the shared library is missing or no CUDA device is present,
+loading or ``Context()`` raises.
+
+Device tensors are passed as objects with ``data_ptr()`` (torch tensors, used
+for device memory and streams only) or as raw integer addresses.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblvspec.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+KERNEL_DEFAULT, KERNEL_SIMT, KERNEL_TCGEN05 = 0, 1, 2
+DEV_WAIT_EXPIRED, DEV_NAN_LOGIT = 0x1, 0x2
+MAX_BATCH, MAX_ROWS, MAX_GAMMA = 128, 128, 64
+
+EXPORTS = (
+    "lvspec_create", "lvspec_destroy", "lvspec_set_stream", "lvspec_device_status",
+    "lvspec_last_error", "lvspec_status_string", "lvspec_launch_count",
+    "lvspec_attention_splits", "lvspec_verify_attention", "lvspec_verify_attention_host",
+    "lvspec_loose_accept", "lvspec_loose_accept_ex", "lvspec_loose_accept_host",
+)
+
+
+class AttnShape(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("batch", "gamma", "n_q_heads", "n_kv_heads", "head_dim", "kv_capacity",
+                 "n_split", "kernel")]
+
+
+class Thresholds(ctypes.Structure):
+    _fields_ = [("lam", ctypes.c_double), ("n_loose", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
+
+
+class LvspecError(RuntimeError):
+    def __init__(self, status: int, text: str):
+        super().__init__(f"lvspec status {status}: {text}")
+        self.status = status
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None) -> ctypes.CDLL:
+    """Loads liblvspec.so; raises OSError when it has not been built."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    path = path or LIB_PATH
+    if not os.path.exists(path):
+        raise OSError(f"{path} not found: build it with "
+                      "`python -m paper_2604_05650_b200.build` (needs nvcc)")
+    lib = ctypes.CDLL(path)
+    vp, i32, u64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint64
+    S = ctypes.POINTER(AttnShape)
+    T = ctypes.POINTER(Thresholds)
+    lib.lvspec_create.argtypes = [ctypes.POINTER(vp), ctypes.c_int]
+    lib.lvspec_destroy.argtypes = [vp]
+    lib.lvspec_set_stream.argtypes = [vp, vp]
+    lib.lvspec_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.lvspec_last_error.argtypes = [vp]
+    lib.lvspec_last_error.restype = ctypes.c_char_p
+    lib.lvspec_status_string.argtypes = [ctypes.c_int]
+    lib.lvspec_status_string.restype = ctypes.c_char_p
+    lib.lvspec_launch_count.argtypes = [vp]
+    lib.lvspec_launch_count.restype = u64
+    lib.lvspec_attention_splits.argtypes = [vp, S, i32]
+    lib.lvspec_attention_splits.restype = i32
+    lib.lvspec_verify_attention.argtypes = [vp, S, vp, vp, vp, vp, vp, vp, vp]
+    lib.lvspec_verify_attention_host.argtypes = [vp, S, vp, vp, vp, vp, vp, vp, vp]
+    lib.lvspec_loose_accept.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp]
+    lib.lvspec_loose_accept_ex.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp, vp, vp]
+    lib.lvspec_loose_accept_host.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp]
+    for name in EXPORTS:
+        fn = getattr(lib, name)
+        if fn.restype is ctypes.c_int and name not in ("lvspec_attention_splits",):
+            fn.restype = ctypes.c_int
+    if path == LIB_PATH:
+        _lib = lib
+    return lib
+
+
+def _addr(x) -> Optional[int]:
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if isinstance(x, np.ndarray):
+        return x.ctypes.data
+    return int(x.data_ptr())
+
+
+def _i32(a: Sequence[int]) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+class Context:
+    """One library context on one CUDA device (``lvspec_create``)."""
+
+    def __init__(self, device: int = 0):
+        self._lib = load_library()
+        h = ctypes.c_void_p()
+        st = self._lib.lvspec_create(ctypes.byref(h), int(device))
+        if st != OK:
+            raise LvspecError(st, self._lib.lvspec_last_error(None).decode())
+        self._h = h
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            self._lib.lvspec_destroy(self._h)
+            self._h = None
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st: int) -> None:
+        if st != OK:
+            raise LvspecError(st, self._lib.lvspec_last_error(self._h).decode())
+
+    def set_stream(self, stream) -> None:
+        """``stream``: a raw cudaStream_t address, or an object with ``cuda_stream``."""
+        s = getattr(stream, "cuda_stream", stream)
+        self._check(self._lib.lvspec_set_stream(self._h, ctypes.c_void_p(int(s) if s else 0)))
+
+    def device_status(self) -> int:
+        flags = ctypes.c_uint32(0)
+        st = self._lib.lvspec_device_status(self._h, ctypes.byref(flags))
+        if st not in (OK, ERR_TIMEOUT):
+            self._check(st)
+        return int(flags.value)
+
+    def launch_count(self) -> int:
+        return int(self._lib.lvspec_launch_count(self._h))
+
+    def attention_splits(self, shape: AttnShape, max_kv_len: int) -> int:
+        return int(self._lib.lvspec_attention_splits(self._h, ctypes.byref(shape), int(max_kv_len)))
+
+    # -- lvspec_verify_attention ------------------------------------------------
+    def verify_attention(self, shape: AttnShape, q, k_cache, v_cache, kv_len, visual_span,
+                         out, visual_mass) -> None:
+        kv_len, span = _i32(kv_len), _i32(visual_span)
+        if kv_len.size != shape.batch or span.size != 2 * shape.batch:
+            raise ValueError("kv_len needs B entries and visual_span B pairs")
+        self._check(self._lib.lvspec_verify_attention(
+            self._h, ctypes.byref(shape), _addr(q), _addr(k_cache), _addr(v_cache),
+            kv_len.ctypes.data, span.ctypes.data, _addr(out), _addr(visual_mass)))
+
+    def verify_attention_host(self, shape: AttnShape, q, k_cache, v_cache, kv_len, visual_span,
+                              out, visual_mass) -> None:
+        kv_len, span = _i32(kv_len), _i32(visual_span)
+        if kv_len.size != shape.batch or span.size != 2 * shape.batch:
+            raise ValueError("kv_len needs B entries and visual_span B pairs")
+        self._check(self._lib.lvspec_verify_attention_host(
+            self._h, ctypes.byref(shape), _addr(q), _addr(k_cache), _addr(v_cache),
+            kv_len.ctypes.data, span.ctypes.data, _addr(out), _addr(visual_mass)))
+
+    # -- lvspec_loose_accept ----------------------------------------------------
+    def loose_accept(self, batch, gamma, vocab, n_mass_heads, target_logits, draft_tokens,
+                     visual_mass, accept_len, shift_window, lam: float = 0.7,
+                     n_loose: int = -1, target_tokens=None, accepted=None) -> None:
+        th = Thresholds(float(lam), int(n_loose), 0)
+        self._check(self._lib.lvspec_loose_accept_ex(
+            self._h, batch, gamma, vocab, n_mass_heads, _addr(target_logits),
+            _addr(draft_tokens), _addr(visual_mass), ctypes.byref(th), int(shift_window),
+            _addr(accept_len), _addr(target_tokens), _addr(accepted)))
+
+    def loose_accept_host(self, batch, gamma, vocab, n_mass_heads, target_logits, draft_tokens,
+                          visual_mass, accept_len, shift_window, lam: float = 0.7,
+                          n_loose: int = -1) -> None:
+        th = Thresholds(float(lam), int(n_loose), 0)
+        self._check(self._lib.lvspec_loose_accept_host(
+            self._h, batch, gamma, vocab, n_mass_heads, _addr(target_logits),
+            _addr(draft_tokens), _addr(visual_mass), ctypes.byref(th), int(shift_window),
+            _addr(accept_len)))
+
+
+HAVE_TCGEN05 = False
+
+
+def available_kernels():
+    """Kernel selectors this build of the library accepts."""
+    return [KERNEL_SIMT, KERNEL_TCGEN05] if HAVE_TCGEN05 else [KERNEL_SIMT]
+
+
+def attn_shape(batch, gamma, n_q_heads, n_kv_heads, head_dim, kv_capacity, n_split=0,
+               kernel=KERNEL_DEFAULT) -> AttnShape:
+    return AttnShape(batch, gamma, n_q_heads, n_kv_heads, head_dim, kv_capacity, n_split, kernel)

@@ -1,0 +1,501 @@
+// Host side of liblvspec.so: context, argument validation, scratch memory and
+// the launch sequence of each call.  Every step of the verify path itself runs
+// in the kernels; nothing here computes on the CPU.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "lvspec_internal.h"
+
+using namespace lvspec;
+
+struct lvspec_ctx {
+    int device = 0;
+    int n_sm = 0;
+    cudaStream_t stream = nullptr;
+    uint32_t *status = nullptr;       // device status word
+    uint32_t *counters = nullptr;     // [LVSPEC_MAX_BATCH] tickets of the acceptance kernel
+    void *scratch = nullptr;          // split partials / argmax partials
+    size_t scratch_bytes = 0;
+    void *staging = nullptr;          // device copies for the *_host calls
+    size_t staging_bytes = 0;
+    uint64_t launches = 0;
+    std::string error;
+};
+
+namespace {
+
+thread_local std::string g_create_error = "no error";
+
+lvspec_status_t fail(lvspec_ctx *ctx, lvspec_status_t st, const std::string &msg)
+{
+    if (ctx) ctx->error = msg;
+    return st;
+}
+
+lvspec_status_t cuda_fail(lvspec_ctx *ctx, const char *what, cudaError_t err)
+{
+    return fail(ctx, LVSPEC_ERR_CUDA,
+                std::string(what) + ": " + cudaGetErrorName(err) + " (" +
+                    cudaGetErrorString(err) + ")");
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+lvspec_status_t ensure(lvspec_ctx *ctx, void **buf, size_t *have, size_t want, bool zero)
+{
+    if (want <= *have) return LVSPEC_OK;
+    if (*buf) {
+        cudaError_t e = cudaStreamSynchronize(ctx->stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, "cudaStreamSynchronize", e);
+        cudaFree(*buf);
+        *buf = nullptr;
+        *have = 0;
+    }
+    size_t bytes = (want + (size_t(1) << 20) - 1) & ~((size_t(1) << 20) - 1);
+    cudaError_t e = cudaMalloc(buf, bytes);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(ctx, LVSPEC_ERR_WORKSPACE,
+                    "scratch allocation of " + std::to_string(bytes) + " bytes failed");
+    }
+    if (zero) {
+        e = cudaMemsetAsync(*buf, 0, bytes, ctx->stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, "cudaMemsetAsync", e);
+    }
+    *have = bytes;
+    return LVSPEC_OK;
+}
+
+int resolve_kernel(const lvspec_attn_shape_t *s)
+{
+    if (s->kernel == LVSPEC_KERNEL_SIMT || s->kernel == LVSPEC_KERNEL_TCGEN05) return s->kernel;
+    return LVSPEC_KERNEL_SIMT;
+}
+
+int choose_splits(const lvspec_ctx *ctx, const lvspec_attn_shape_t *s, int max_kv_len)
+{
+    const int tiles = (max_kv_len + 127) / 128;           // splits never go below 128 positions
+    const int units = s->batch * s->n_kv_heads;
+    int want = (2 * ctx->n_sm + units - 1) / units;        // about two CTAs per SM
+    if (want < 1) want = 1;
+    if (want > tiles) want = tiles;
+    if (want > 256) want = 256;
+    return want;
+}
+
+// Validation shared by the device and host forms.  On success fills seq.
+lvspec_status_t check_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, const void *q,
+                                const void *k, const void *v, const int32_t *kv_len,
+                                const int32_t *span, const void *out, const float *mass,
+                                bool device_ptrs, SeqInfo *seq, int *max_len)
+{
+    if (!ctx) return LVSPEC_ERR_INVALID_ARG;
+    if (!s || !q || !k || !v || !kv_len || !span || !out || !mass)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "null argument");
+    if (s->batch < 1 || s->batch > LVSPEC_MAX_BATCH)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "batch outside 1..LVSPEC_MAX_BATCH");
+    if (s->gamma < 1 || s->gamma > LVSPEC_MAX_GAMMA)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "gamma outside 1..LVSPEC_MAX_GAMMA");
+    if (s->n_kv_heads < 1 || s->n_q_heads < 1 || s->n_q_heads % s->n_kv_heads != 0)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "n_q_heads must be a positive multiple of n_kv_heads");
+    if (s->n_kv_heads > 65535)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "n_kv_heads beyond 65535");
+    if (s->kv_capacity < 1) return fail(ctx, LVSPEC_ERR_INVALID_ARG, "kv_capacity < 1");
+    if (s->n_split < 0 || s->n_split > 1024)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "n_split outside 0..1024");
+    if (s->kernel < 0 || s->kernel > LVSPEC_KERNEL_TCGEN05)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "unknown kernel selector");
+    if (s->head_dim != 64 && s->head_dim != 128)
+        return fail(ctx, LVSPEC_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+    const int G = s->n_q_heads / s->n_kv_heads;
+    if ((long long)s->gamma * G > LVSPEC_MAX_ROWS)
+        return fail(ctx, LVSPEC_ERR_UNSUPPORTED,
+                    "gamma * (n_q_heads / n_kv_heads) beyond LVSPEC_MAX_ROWS");
+    if (device_ptrs && (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) ||
+                        (reinterpret_cast<uintptr_t>(mass) & 3u)))
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "device tensors must be 16-byte aligned");
+    int mx = 0;
+    for (int b = 0; b < s->batch; ++b) {
+        const int L = kv_len[b], vs = span[2 * b], ve = span[2 * b + 1];
+        if (L < s->gamma || L > s->kv_capacity)
+            return fail(ctx, LVSPEC_ERR_INVALID_ARG,
+                        "kv_len[" + std::to_string(b) + "] outside gamma..kv_capacity");
+        if (vs < 0 || vs > ve || ve > L - s->gamma)
+            return fail(ctx, LVSPEC_ERR_INVALID_ARG,
+                        "visual_span[" + std::to_string(b) + "] outside 0..kv_len-gamma");
+        seq->kv_len[b] = L;
+        seq->span_start[b] = vs;
+        seq->span_end[b] = ve;
+        if (L > mx) mx = L;
+    }
+    *max_len = mx;
+    return LVSPEC_OK;
+}
+
+lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, const SeqInfo &seq,
+                              int max_len, const void *q, const void *k, const void *v, void *out,
+                              float *mass)
+{
+    AttnParams p;
+    std::memset(&p, 0, sizeof p);
+    p.q = static_cast<const uint16_t *>(q);
+    p.k = static_cast<const uint16_t *>(k);
+    p.v = static_cast<const uint16_t *>(v);
+    p.out = static_cast<uint16_t *>(out);
+    p.mass = mass;
+    p.status = ctx->status;
+    p.B = s->batch;
+    p.gamma = s->gamma;
+    p.Hq = s->n_q_heads;
+    p.Hkv = s->n_kv_heads;
+    p.D = s->head_dim;
+    p.Lmax = s->kv_capacity;
+    p.G = p.Hq / p.Hkv;
+    p.M = p.gamma * p.G;
+    p.n_split = s->n_split > 0 ? s->n_split : choose_splits(ctx, s, max_len);
+    p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)p.D));
+
+    const size_t o_bytes = part_o_elems(p) * sizeof(float);
+    const size_t st_bytes = part_stat_elems(p) * sizeof(float);
+    lvspec_status_t st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, o_bytes + st_bytes, false);
+    if (st != LVSPEC_OK) return st;
+    p.part_o = static_cast<float *>(ctx->scratch);
+    p.part_stat = reinterpret_cast<float *>(static_cast<char *>(ctx->scratch) + o_bytes);
+
+    int launches = 0;
+    cudaError_t e;
+    const int kernel = resolve_kernel(s);
+    if (kernel == LVSPEC_KERNEL_TCGEN05)
+        return fail(ctx, LVSPEC_ERR_UNSUPPORTED, "tcgen05 kernel not built");
+    e = launch_attn_simt(p, seq, ctx->stream, &launches);
+    ctx->launches += launches;
+    if (e != cudaSuccess) return cuda_fail(ctx, "attention kernel launch", e);
+    launches = 0;
+    e = launch_attn_combine(p, ctx->stream, &launches);
+    ctx->launches += launches;
+    if (e != cudaSuccess) return cuda_fail(ctx, "combine kernel launch", e);
+    return LVSPEC_OK;
+}
+
+lvspec_status_t check_accept(lvspec_ctx *ctx, int batch, int gamma, int vocab, int heads,
+                             const void *logits, const void *draft, const void *mass,
+                             const lvspec_thresholds_t *th, int window, const void *accept_len,
+                             bool device_ptrs, int *n_loose)
+{
+    if (!ctx) return LVSPEC_ERR_INVALID_ARG;
+    if (!logits || !draft || !mass || !th || !accept_len)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "null argument");
+    if (batch < 1 || batch > LVSPEC_MAX_BATCH)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "batch outside 1..LVSPEC_MAX_BATCH");
+    if (gamma < 1 || gamma > LVSPEC_MAX_GAMMA)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "gamma outside 1..LVSPEC_MAX_GAMMA");
+    if (vocab < 1) return fail(ctx, LVSPEC_ERR_INVALID_ARG, "vocab < 1");
+    if (heads < 1) return fail(ctx, LVSPEC_ERR_INVALID_ARG, "n_mass_heads < 1");
+    if (window < 0) return fail(ctx, LVSPEC_ERR_INVALID_ARG, "shift_window < 0");
+    if (device_ptrs && ((reinterpret_cast<uintptr_t>(logits) & 3u) ||
+                        (reinterpret_cast<uintptr_t>(draft) & 3u) ||
+                        (reinterpret_cast<uintptr_t>(mass) & 3u) ||
+                        (reinterpret_cast<uintptr_t>(accept_len) & 3u)))
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "misaligned device pointer");
+    int n = th->n_loose;
+    if (n < 0) {
+        if (!(th->lambda >= 0.0 && th->lambda <= 1.0))
+            return fail(ctx, LVSPEC_ERR_INVALID_ARG, "lambda outside [0, 1]");
+        n = (int)std::floor(th->lambda * (double)gamma + 1e-9);
+    }
+    if (n > gamma) return fail(ctx, LVSPEC_ERR_INVALID_ARG, "n_loose > gamma");
+    *n_loose = n;
+    return LVSPEC_OK;
+}
+
+lvspec_status_t run_accept(lvspec_ctx *ctx, int batch, int gamma, int vocab, int heads,
+                           const float *logits, const int32_t *draft, const float *mass,
+                           int n_loose, int window, int32_t *accept_len, int32_t *target,
+                           uint8_t *accepted)
+{
+    AcceptParams p;
+    std::memset(&p, 0, sizeof p);
+    p.logits = logits;
+    p.draft = draft;
+    p.mass = mass;
+    p.accept_len = accept_len;
+    p.target = target;
+    p.accepted = accepted;
+    p.counters = ctx->counters;
+    p.status = ctx->status;
+    p.B = batch;
+    p.gamma = gamma;
+    p.V = vocab;
+    p.Hm = heads;
+    p.n_loose = n_loose;
+    p.window = window > gamma ? gamma : window;
+    // slices: enough CTAs for two per SM, at least 4096 elements each
+    int rows = batch * gamma;
+    int vs = (2 * ctx->n_sm + rows - 1) / rows;
+    const int max_vs = (vocab + 4095) / 4096;
+    if (vs > max_vs) vs = max_vs;
+    if (vs < 1) vs = 1;
+    p.n_vsplit = vs;
+    const size_t n_part = (size_t)rows * vs;
+    lvspec_status_t st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes,
+                                n_part * (sizeof(float) + sizeof(int32_t)), false);
+    if (st != LVSPEC_OK) return st;
+    p.part_val = static_cast<float *>(ctx->scratch);
+    p.part_idx = reinterpret_cast<int32_t *>(p.part_val + n_part);
+    int launches = 0;
+    cudaError_t e = launch_loose_accept(p, ctx->stream, &launches);
+    ctx->launches += launches;
+    if (e != cudaSuccess) return cuda_fail(ctx, "acceptance kernel launch", e);
+    return LVSPEC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+lvspec_status_t lvspec_create(lvspec_ctx_t **out, int device)
+{
+    if (!out) {
+        g_create_error = "null context pointer";
+        return LVSPEC_ERR_INVALID_ARG;
+    }
+    *out = nullptr;
+    int n_dev = 0;
+    cudaError_t e = cudaGetDeviceCount(&n_dev);
+    if (e != cudaSuccess || n_dev == 0) {
+        cudaGetLastError();
+        g_create_error = std::string("no CUDA device: ") + cudaGetErrorString(e);
+        return LVSPEC_ERR_CUDA;
+    }
+    if (device < 0 || device >= n_dev) {
+        g_create_error = "device ordinal out of range";
+        return LVSPEC_ERR_INVALID_ARG;
+    }
+    lvspec_ctx *ctx = new (std::nothrow) lvspec_ctx();
+    if (!ctx) {
+        g_create_error = "out of host memory";
+        return LVSPEC_ERR_WORKSPACE;
+    }
+    ctx->device = device;
+    ctx->error = "no error";
+    cudaDeviceProp prop;
+    if ((e = cudaSetDevice(device)) != cudaSuccess ||
+        (e = cudaGetDeviceProperties(&prop, device)) != cudaSuccess) {
+        g_create_error = std::string("cudaSetDevice: ") + cudaGetErrorString(e);
+        delete ctx;
+        return LVSPEC_ERR_CUDA;
+    }
+    if (prop.major != 10) {
+        g_create_error = "this library holds sm_100a code only; device is sm_" +
+                         std::to_string(prop.major) + std::to_string(prop.minor);
+        delete ctx;
+        return LVSPEC_ERR_UNSUPPORTED;
+    }
+    ctx->n_sm = prop.multiProcessorCount;
+    const size_t small = sizeof(uint32_t) * (1 + LVSPEC_MAX_BATCH);
+    if ((e = cudaMalloc(reinterpret_cast<void **>(&ctx->status), small)) != cudaSuccess ||
+        (e = cudaMemset(ctx->status, 0, small)) != cudaSuccess) {
+        g_create_error = std::string("status allocation: ") + cudaGetErrorString(e);
+        delete ctx;
+        return LVSPEC_ERR_WORKSPACE;
+    }
+    ctx->counters = ctx->status + 1;
+    lvspec_status_t st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, size_t(8) << 20, true);
+    if (st != LVSPEC_OK) {
+        g_create_error = ctx->error;
+        cudaFree(ctx->status);
+        delete ctx;
+        return st;
+    }
+    cudaDeviceSynchronize();
+    *out = ctx;
+    return LVSPEC_OK;
+}
+
+lvspec_status_t lvspec_destroy(lvspec_ctx_t *ctx)
+{
+    if (!ctx) return LVSPEC_ERR_INVALID_ARG;
+    cudaSetDevice(ctx->device);
+    cudaStreamSynchronize(ctx->stream);
+    cudaFree(ctx->scratch);
+    cudaFree(ctx->staging);
+    cudaFree(ctx->status);
+    delete ctx;
+    return LVSPEC_OK;
+}
+
+lvspec_status_t lvspec_set_stream(lvspec_ctx_t *ctx, void *cuda_stream)
+{
+    if (!ctx) return LVSPEC_ERR_INVALID_ARG;
+    ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    return LVSPEC_OK;
+}
+
+lvspec_status_t lvspec_device_status(lvspec_ctx_t *ctx, uint32_t *flags)
+{
+    if (!ctx || !flags) return LVSPEC_ERR_INVALID_ARG;
+    cudaSetDevice(ctx->device);
+    uint32_t h = 0;
+    cudaError_t e = cudaMemcpyAsync(&h, ctx->status, sizeof h, cudaMemcpyDeviceToHost, ctx->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->status, 0, sizeof h, ctx->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, "reading the device status", e);
+    *flags = h;
+    if (h & LVSPEC_DEV_WAIT_EXPIRED)
+        return fail(ctx, LVSPEC_ERR_TIMEOUT, "a bounded device-side wait ran out");
+    return LVSPEC_OK;
+}
+
+const char *lvspec_last_error(const lvspec_ctx_t *ctx)
+{
+    return ctx ? ctx->error.c_str() : g_create_error.c_str();
+}
+
+const char *lvspec_status_string(lvspec_status_t status)
+{
+    switch (status) {
+        case LVSPEC_OK: return "ok";
+        case LVSPEC_ERR_INVALID_ARG: return "invalid argument";
+        case LVSPEC_ERR_UNSUPPORTED: return "unsupported shape";
+        case LVSPEC_ERR_WORKSPACE: return "scratch memory allocation failed";
+        case LVSPEC_ERR_CUDA: return "CUDA error";
+        case LVSPEC_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+uint64_t lvspec_launch_count(const lvspec_ctx_t *ctx) { return ctx ? ctx->launches : 0; }
+
+int32_t lvspec_attention_splits(const lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                int32_t max_kv_len)
+{
+    if (!ctx || !shape || shape->batch < 1 || shape->n_kv_heads < 1 || max_kv_len < 1) return 0;
+    return shape->n_split > 0 ? shape->n_split : choose_splits(ctx, shape, max_kv_len);
+}
+
+lvspec_status_t lvspec_verify_attention(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                        const void *q, const void *k_cache, const void *v_cache,
+                                        const int32_t *kv_len, const int32_t *visual_span,
+                                        void *out, float *visual_mass)
+{
+    SeqInfo seq;
+    int max_len = 0;
+    lvspec_status_t st = check_attention(ctx, shape, q, k_cache, v_cache, kv_len, visual_span, out,
+                                         visual_mass, true, &seq, &max_len);
+    if (st != LVSPEC_OK) return st;
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
+    return run_attention(ctx, shape, seq, max_len, q, k_cache, v_cache, out, visual_mass);
+}
+
+lvspec_status_t lvspec_verify_attention_host(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                             const void *q, const void *k_cache,
+                                             const void *v_cache, const int32_t *kv_len,
+                                             const int32_t *visual_span, void *out,
+                                             float *visual_mass)
+{
+    SeqInfo seq;
+    int max_len = 0;
+    lvspec_status_t st = check_attention(ctx, shape, q, k_cache, v_cache, kv_len, visual_span, out,
+                                         visual_mass, false, &seq, &max_len);
+    if (st != LVSPEC_OK) return st;
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
+    auto up = [](size_t x) { return (x + 255) & ~size_t(255); };
+    const size_t q_bytes = (size_t)shape->batch * shape->gamma * shape->n_q_heads * shape->head_dim * 2;
+    const size_t kv_bytes = (size_t)shape->batch * shape->n_kv_heads * shape->kv_capacity * shape->head_dim * 2;
+    const size_t m_bytes = (size_t)shape->batch * shape->gamma * shape->n_q_heads * sizeof(float);
+    const size_t total = 2 * up(q_bytes) + 2 * up(kv_bytes) + up(m_bytes);
+    st = ensure(ctx, &ctx->staging, &ctx->staging_bytes, total, false);
+    if (st != LVSPEC_OK) return st;
+    char *base = static_cast<char *>(ctx->staging);
+    char *dq = base, *dk = dq + up(q_bytes), *dv = dk + up(kv_bytes), *dout = dv + up(kv_bytes),
+         *dm = dout + up(q_bytes);
+    if ((e = cudaMemcpyAsync(dq, q, q_bytes, cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(dk, k_cache, kv_bytes, cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(dv, v_cache, kv_bytes, cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess)
+        return cuda_fail(ctx, "host to device copy", e);
+    st = run_attention(ctx, shape, seq, max_len, dq, dk, dv, dout, reinterpret_cast<float *>(dm));
+    if (st != LVSPEC_OK) return st;
+    if ((e = cudaMemcpyAsync(out, dout, q_bytes, cudaMemcpyDeviceToHost, ctx->stream)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(visual_mass, dm, m_bytes, cudaMemcpyDeviceToHost, ctx->stream)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(ctx->stream)) != cudaSuccess)
+        return cuda_fail(ctx, "device to host copy", e);
+    return LVSPEC_OK;
+}
+
+lvspec_status_t lvspec_loose_accept_ex(lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,
+                                       int32_t vocab, int32_t n_mass_heads,
+                                       const float *target_logits, const int32_t *draft_tokens,
+                                       const float *visual_mass,
+                                       const lvspec_thresholds_t *thresholds,
+                                       int32_t shift_window, int32_t *accept_len,
+                                       int32_t *target_tokens, uint8_t *accepted)
+{
+    int n_loose = 0;
+    lvspec_status_t st = check_accept(ctx, batch, gamma, vocab, n_mass_heads, target_logits,
+                                      draft_tokens, visual_mass, thresholds, shift_window,
+                                      accept_len, true, &n_loose);
+    if (st != LVSPEC_OK) return st;
+    if (target_tokens && (reinterpret_cast<uintptr_t>(target_tokens) & 3u))
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "misaligned device pointer");
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
+    return run_accept(ctx, batch, gamma, vocab, n_mass_heads, target_logits, draft_tokens,
+                      visual_mass, n_loose, shift_window, accept_len, target_tokens, accepted);
+}
+
+lvspec_status_t lvspec_loose_accept(lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,
+                                    int32_t vocab, int32_t n_mass_heads,
+                                    const float *target_logits, const int32_t *draft_tokens,
+                                    const float *visual_mass,
+                                    const lvspec_thresholds_t *thresholds, int32_t shift_window,
+                                    int32_t *accept_len)
+{
+    return lvspec_loose_accept_ex(ctx, batch, gamma, vocab, n_mass_heads, target_logits,
+                                  draft_tokens, visual_mass, thresholds, shift_window, accept_len,
+                                  nullptr, nullptr);
+}
+
+lvspec_status_t lvspec_loose_accept_host(lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,
+                                         int32_t vocab, int32_t n_mass_heads,
+                                         const float *target_logits, const int32_t *draft_tokens,
+                                         const float *visual_mass,
+                                         const lvspec_thresholds_t *thresholds,
+                                         int32_t shift_window, int32_t *accept_len)
+{
+    int n_loose = 0;
+    lvspec_status_t st = check_accept(ctx, batch, gamma, vocab, n_mass_heads, target_logits,
+                                      draft_tokens, visual_mass, thresholds, shift_window,
+                                      accept_len, false, &n_loose);
+    if (st != LVSPEC_OK) return st;
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
+    auto up = [](size_t x) { return (x + 255) & ~size_t(255); };
+    const size_t lg_bytes = (size_t)batch * gamma * vocab * sizeof(float);
+    const size_t dr_bytes = (size_t)batch * gamma * sizeof(int32_t);
+    const size_t ms_bytes = (size_t)batch * gamma * n_mass_heads * sizeof(float);
+    const size_t al_bytes = (size_t)batch * sizeof(int32_t);
+    st = ensure(ctx, &ctx->staging, &ctx->staging_bytes,
+                up(lg_bytes) + up(dr_bytes) + up(ms_bytes) + up(al_bytes), false);
+    if (st != LVSPEC_OK) return st;
+    char *dl = static_cast<char *>(ctx->staging), *dd = dl + up(lg_bytes), *dm = dd + up(dr_bytes),
+         *da = dm + up(ms_bytes);
+    if ((e = cudaMemcpyAsync(dl, target_logits, lg_bytes, cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(dd, draft_tokens, dr_bytes, cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(dm, visual_mass, ms_bytes, cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess)
+        return cuda_fail(ctx, "host to device copy", e);
+    st = run_accept(ctx, batch, gamma, vocab, n_mass_heads, reinterpret_cast<float *>(dl),
+                    reinterpret_cast<int32_t *>(dd), reinterpret_cast<float *>(dm), n_loose,
+                    shift_window, reinterpret_cast<int32_t *>(da), nullptr, nullptr);
+    if (st != LVSPEC_OK) return st;
+    if ((e = cudaMemcpyAsync(accept_len, da, al_bytes, cudaMemcpyDeviceToHost, ctx->stream)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(ctx->stream)) != cudaSuccess)
+        return cuda_fail(ctx, "device to host copy", e);
+    return LVSPEC_OK;
+}
+
+}  // extern "C"

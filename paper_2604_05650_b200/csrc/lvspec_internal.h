@@ -1,0 +1,60 @@
+// Internal declarations shared by the translation units of liblvspec.so.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lvspec.h"
+
+namespace lvspec {
+
+// Per-sequence lengths travel as kernel parameters (the C ABI takes them as
+// host arrays), so a launch needs no host->device copy of its own.
+struct SeqInfo {
+    int32_t kv_len[LVSPEC_MAX_BATCH];
+    int32_t span_start[LVSPEC_MAX_BATCH];
+    int32_t span_end[LVSPEC_MAX_BATCH];
+};
+
+struct AttnParams {
+    const uint16_t *q;     // [B, gamma, Hq, D] bf16
+    const uint16_t *k;     // [B, Hkv, Lmax, D] bf16
+    const uint16_t *v;
+    uint16_t *out;         // [B, gamma, Hq, D] bf16
+    float *mass;           // [B, gamma, Hq]
+    float *part_o;         // [B, Hkv, n_split, M, D] fp32, unnormalised
+    float *part_stat;      // [B, Hkv, n_split, M, 4]: m (log2 units), l, l_vis, unused
+    uint32_t *status;      // device status word
+    int32_t B, gamma, Hq, Hkv, D, Lmax, G, M, n_split;
+    float scale_log2;      // log2(e) / sqrt(D)
+};
+
+// Partial results of one KV split, rows r = g * G + hg.
+static inline size_t part_o_elems(const AttnParams &p)
+{
+    return (size_t)p.B * p.Hkv * p.n_split * p.M * p.D;
+}
+static inline size_t part_stat_elems(const AttnParams &p)
+{
+    return (size_t)p.B * p.Hkv * p.n_split * p.M * 4;
+}
+
+cudaError_t launch_attn_simt(const AttnParams &p, const SeqInfo &seq, cudaStream_t stream,
+                             int *launches);
+cudaError_t launch_attn_combine(const AttnParams &p, cudaStream_t stream, int *launches);
+
+struct AcceptParams {
+    const float *logits;      // [B, gamma, V]
+    const int32_t *draft;     // [B, gamma]
+    const float *mass;        // [B, gamma, Hm]
+    int32_t *accept_len;      // [B]
+    int32_t *target;          // optional [B, gamma]
+    uint8_t *accepted;        // optional [B, gamma]
+    float *part_val;          // [B, gamma, n_vsplit]
+    int32_t *part_idx;        // [B, gamma, n_vsplit]
+    uint32_t *counters;       // [B], zero between calls
+    uint32_t *status;
+    int32_t B, gamma, V, Hm, n_loose, window, n_vsplit;
+};
+cudaError_t launch_loose_accept(const AcceptParams &p, cudaStream_t stream, int *launches);
+
+}  // namespace lvspec

@@ -1,0 +1,260 @@
+// Verification attention with fused visual mass, CUDA-core (SIMT) kernel, and
+// the split-KV combine kernel.  Covers every supported shape; it is the plain
+// device implementation the tensor-core kernel is cross-checked with.
+//
+// One CTA owns one KV split of one (sequence, KV head) and all M = gamma * G
+// query rows that read that head (row r = g * G + hg).  Per tile of 32 cache
+// positions: scores by fp32 FMA from shared memory, an online softmax per row
+// (fp32, base-2 exponent), the running sums l and l_vis (probability mass
+// inside the visual span) and the P.V update.  The unnormalised partials go to
+// scratch memory; `attn_combine_kernel` merges the splits.
+#include <cuda_bf16.h>
+
+#include "lvspec_internal.h"
+
+namespace lvspec {
+namespace {
+
+constexpr int kTile = 32;      // cache positions per tile
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b)
+{
+    return __uint_as_float(((uint32_t)b) << 16);
+}
+
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads)
+attn_simt_kernel(const AttnParams p, const SeqInfo seq)
+{
+    constexpr int DP = D + 4;                 // padded row: conflict-free float4 reads
+    constexpr int D4 = D / 4;
+    constexpr int kRowGroups = kThreads / D4; // thread (rg, d4) accumulates rows rg, rg+kRowGroups, ...
+    constexpr int kMaxRowsPerThread = (LVSPEC_MAX_ROWS + kRowGroups - 1) / kRowGroups;
+
+    extern __shared__ __align__(16) float smem[];
+    const int M = p.M;
+    float *q_s = smem;                        // [M][DP]
+    float *k_s = q_s + (size_t)M * DP;        // [kTile][DP]
+    float *v_s = k_s + kTile * DP;            // [kTile][DP]
+    float *s_s = v_s + kTile * DP;            // [M][kTile]  scores, then probabilities
+    float *m_s = s_s + (size_t)M * kTile;     // [M]
+    float *l_s = m_s + M;
+    float *lv_s = l_s + M;
+    float *corr_s = lv_s + M;
+
+    const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int L = seq.kv_len[b];
+    const int vs = seq.span_start[b], ve = seq.span_end[b];
+    const int G = p.G, gamma = p.gamma;
+
+    // split ranges are whole tiles
+    const int n_tiles = (L + kTile - 1) / kTile;
+    const int tiles_per_split = (n_tiles + p.n_split - 1) / p.n_split;
+    const int t_begin = split * tiles_per_split;
+    const int t_end = min(n_tiles, t_begin + tiles_per_split);
+
+    // Q rows of this KV head -> shared memory as fp32
+    for (int i = tid; i < M * D; i += kThreads) {
+        const int r = i / D, d = i - r * D;
+        const int g = r / G, hg = r - g * G;
+        const size_t off = (((size_t)b * gamma + g) * p.Hq + kvh * G + hg) * D + d;
+        q_s[r * DP + d] = bf16_bits_to_float(p.q[off]);
+    }
+    for (int r = tid; r < M; r += kThreads) {
+        m_s[r] = -INFINITY;
+        l_s[r] = 0.f;
+        lv_s[r] = 0.f;
+    }
+
+    const int d4 = tid % D4, rg = tid / D4;
+    float4 acc[kMaxRowsPerThread];
+#pragma unroll
+    for (int i = 0; i < kMaxRowsPerThread; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+    const uint16_t *kbase = p.k + ((size_t)b * p.Hkv + kvh) * (size_t)p.Lmax * D;
+    const uint16_t *vbase = p.v + ((size_t)b * p.Hkv + kvh) * (size_t)p.Lmax * D;
+    __syncthreads();
+
+    for (int t = t_begin; t < t_end; ++t) {
+        const int pos0 = t * kTile;
+        // K and V tile -> shared memory (8 bf16 per 16-byte load)
+        for (int i = tid; i < kTile * (D / 8); i += kThreads) {
+            const int j = i / (D / 8), c = i - j * (D / 8);
+            const int pos = pos0 + j;
+            uint4 kk = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
+            if (pos < L) {
+                kk = *reinterpret_cast<const uint4 *>(kbase + (size_t)pos * D + c * 8);
+                vv = *reinterpret_cast<const uint4 *>(vbase + (size_t)pos * D + c * 8);
+            }
+            const uint32_t kw[4] = {kk.x, kk.y, kk.z, kk.w}, vw[4] = {vv.x, vv.y, vv.z, vv.w};
+            float *kd = k_s + j * DP + c * 8, *vd = v_s + j * DP + c * 8;
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+                kd[2 * w] = __uint_as_float(kw[w] << 16);
+                kd[2 * w + 1] = __uint_as_float(kw[w] & 0xffff0000u);
+                vd[2 * w] = __uint_as_float(vw[w] << 16);
+                vd[2 * w + 1] = __uint_as_float(vw[w] & 0xffff0000u);
+            }
+        }
+        __syncthreads();
+
+        // scores: s[r][j], one (r, j) pair per thread per pass
+        for (int i = tid; i < M * kTile; i += kThreads) {
+            const int r = i / kTile, j = i - r * kTile;
+            const float4 *qr = reinterpret_cast<const float4 *>(q_s + r * DP);
+            const float4 *kr = reinterpret_cast<const float4 *>(k_s + j * DP);
+            float s = 0.f;
+#pragma unroll 8
+            for (int c = 0; c < D4; ++c) {
+                const float4 a = qr[c], k4 = kr[c];
+                s = fmaf(a.x, k4.x, s);
+                s = fmaf(a.y, k4.y, s);
+                s = fmaf(a.z, k4.z, s);
+                s = fmaf(a.w, k4.w, s);
+            }
+            s_s[i] = s * p.scale_log2;
+        }
+        __syncthreads();
+
+        // online softmax, one warp per row, lane = position inside the tile
+        for (int r = warp; r < M; r += kThreads / 32) {
+            const int g = r / G;
+            const int pos = pos0 + lane;
+            const bool visible = pos < L - gamma + g + 1;
+            const float s = visible ? s_s[r * kTile + lane] : -INFINITY;
+            float mx = s;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            const float m_old = m_s[r];
+            const float m_new = fmaxf(m_old, mx);
+            float pr = 0.f, corr = 1.f;
+            if (m_new > -INFINITY) {
+                pr = visible ? fast_exp2(s - m_new) : 0.f;
+                corr = fast_exp2(m_old - m_new);  // m_old = -inf gives 0
+            }
+            float sum = pr, sumv = (pos >= vs && pos < ve) ? pr : 0.f;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                sum += __shfl_xor_sync(0xffffffffu, sum, o);
+                sumv += __shfl_xor_sync(0xffffffffu, sumv, o);
+            }
+            s_s[r * kTile + lane] = pr;
+            if (lane == 0) {
+                m_s[r] = m_new;
+                l_s[r] = l_s[r] * corr + sum;
+                lv_s[r] = lv_s[r] * corr + sumv;
+                corr_s[r] = corr;
+            }
+        }
+        __syncthreads();
+
+        // O[r][:] = O[r][:] * corr + sum_j p[r][j] * V[j][:]
+#pragma unroll
+        for (int i = 0; i < kMaxRowsPerThread; ++i) {
+            const int r = rg + i * kRowGroups;
+            if (r < M) {
+                const float c = corr_s[r];
+                float4 a = acc[i];
+                a.x *= c; a.y *= c; a.z *= c; a.w *= c;
+                const float *pr = s_s + r * kTile;
+#pragma unroll 8
+                for (int j = 0; j < kTile; ++j) {
+                    const float pj = pr[j];
+                    const float4 v4 = *reinterpret_cast<const float4 *>(v_s + j * DP + d4 * 4);
+                    a.x = fmaf(pj, v4.x, a.x);
+                    a.y = fmaf(pj, v4.y, a.y);
+                    a.z = fmaf(pj, v4.z, a.z);
+                    a.w = fmaf(pj, v4.w, a.w);
+                }
+                acc[i] = a;
+            }
+        }
+        __syncthreads();
+    }
+
+    // partials of this split
+    const size_t unit = ((size_t)b * p.Hkv + kvh) * p.n_split + split;
+    float *po = p.part_o + unit * (size_t)M * D;
+#pragma unroll
+    for (int i = 0; i < kMaxRowsPerThread; ++i) {
+        const int r = rg + i * kRowGroups;
+        if (r < M) *reinterpret_cast<float4 *>(po + (size_t)r * D + d4 * 4) = acc[i];
+    }
+    float *ps = p.part_stat + unit * (size_t)M * 4;
+    for (int r = tid; r < M; r += kThreads)
+        *reinterpret_cast<float4 *>(ps + r * 4) = make_float4(m_s[r], l_s[r], lv_s[r], 0.f);
+}
+
+// Merge of the KV splits: one CTA per (sequence, KV head, row), one thread per
+// output channel.  Splits are merged in index order, so the result does not
+// depend on scheduling.
+__global__ void attn_combine_kernel(const AttnParams p)
+{
+    const int r = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+    const int d = threadIdx.x;
+    const int M = p.M, D = p.D, ns = p.n_split;
+    const size_t unit0 = ((size_t)b * p.Hkv + kvh) * ns;
+    const float *ps = p.part_stat + unit0 * (size_t)M * 4 + r * 4;
+
+    float m_star = -INFINITY;
+    for (int s = 0; s < ns; ++s) m_star = fmaxf(m_star, ps[(size_t)s * M * 4]);
+    float l = 0.f, lv = 0.f, o = 0.f;
+    for (int s = 0; s < ns; ++s) {
+        const float4 st = *reinterpret_cast<const float4 *>(ps + (size_t)s * M * 4);
+        if (st.y > 0.f) {
+            const float w = exp2f(st.x - m_star);
+            l = fmaf(w, st.y, l);
+            lv = fmaf(w, st.z, lv);
+            o = fmaf(w, p.part_o[((unit0 + s) * (size_t)M + r) * D + d], o);
+        }
+    }
+    const float inv = 1.f / l;
+    const int g = r / p.G, hg = r - g * p.G;
+    const size_t row = ((size_t)b * p.gamma + g) * p.Hq + kvh * p.G + hg;
+    reinterpret_cast<__nv_bfloat16 *>(p.out)[row * D + d] = __float2bfloat16_rn(o * inv);
+    if (d == 0) p.mass[row] = lv * inv;
+}
+
+}  // namespace
+
+cudaError_t launch_attn_simt(const AttnParams &p, const SeqInfo &seq, cudaStream_t stream,
+                             int *launches)
+{
+    const int DP = p.D + 4;
+    const size_t smem = sizeof(float) * ((size_t)p.M * DP + 2 * kTile * DP + (size_t)p.M * kTile +
+                                         4 * (size_t)p.M);
+    dim3 grid(p.n_split, p.Hkv, p.B);
+    cudaError_t err;
+    if (p.D == 128) {
+        err = cudaFuncSetAttribute(attn_simt_kernel<128>,
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        attn_simt_kernel<128><<<grid, kThreads, smem, stream>>>(p, seq);
+    } else {
+        err = cudaFuncSetAttribute(attn_simt_kernel<64>,
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        attn_simt_kernel<64><<<grid, kThreads, smem, stream>>>(p, seq);
+    }
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_attn_combine(const AttnParams &p, cudaStream_t stream, int *launches)
+{
+    dim3 grid(p.M, p.Hkv, p.B);
+    attn_combine_kernel<<<grid, p.D, 0, stream>>>(p);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace lvspec
