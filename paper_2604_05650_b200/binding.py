@@ -152,7 +152,7 @@ class Context:
     def verify_attention(self, shape: AttnShape, q, k_cache, v_cache, kv_len, visual_span,
                          out, visual_mass) -> None:
         kv_len, span = _i32(kv_len), _i32(visual_span)
-        if kv_len.size != shape.batch or span.size != 2 * shape.batch:
+        if shape.batch >= 1 and (kv_len.size != shape.batch or span.size != 2 * shape.batch):
             raise ValueError("kv_len needs B entries and visual_span B pairs")
         self._check(self._lib.lvspec_verify_attention(
             self._h, ctypes.byref(shape), _addr(q), _addr(k_cache), _addr(v_cache),
@@ -161,7 +161,7 @@ class Context:
     def verify_attention_host(self, shape: AttnShape, q, k_cache, v_cache, kv_len, visual_span,
                               out, visual_mass) -> None:
         kv_len, span = _i32(kv_len), _i32(visual_span)
-        if kv_len.size != shape.batch or span.size != 2 * shape.batch:
+        if shape.batch >= 1 and (kv_len.size != shape.batch or span.size != 2 * shape.batch):
             raise ValueError("kv_len needs B entries and visual_span B pairs")
         self._check(self._lib.lvspec_verify_attention_host(
             self._h, ctypes.byref(shape), _addr(q), _addr(k_cache), _addr(v_cache),
