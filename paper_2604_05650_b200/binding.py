@@ -187,7 +187,7 @@ class Context:
             _addr(accept_len)))
 
 
-HAVE_TCGEN05 = False
+HAVE_TCGEN05 = True
 
 
 def available_kernels():

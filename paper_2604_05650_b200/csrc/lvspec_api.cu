@@ -69,17 +69,28 @@ lvspec_status_t ensure(lvspec_ctx *ctx, void **buf, size_t *have, size_t want, b
     return LVSPEC_OK;
 }
 
+// The tensor-core kernel covers head_dim 128 with at least one full tile of
+// cache; everything else runs on the CUDA-core kernel.
+bool tc_shape(const lvspec_attn_shape_t *s)
+{
+    return s->head_dim == 128 && s->kv_capacity >= 128;
+}
+
 int resolve_kernel(const lvspec_attn_shape_t *s)
 {
     if (s->kernel == LVSPEC_KERNEL_SIMT || s->kernel == LVSPEC_KERNEL_TCGEN05) return s->kernel;
-    return LVSPEC_KERNEL_SIMT;
+    return tc_shape(s) ? LVSPEC_KERNEL_TCGEN05 : LVSPEC_KERNEL_SIMT;
 }
 
 int choose_splits(const lvspec_ctx *ctx, const lvspec_attn_shape_t *s, int max_kv_len)
 {
     const int tiles = (max_kv_len + 127) / 128;           // splits never go below 128 positions
     const int units = s->batch * s->n_kv_heads;
-    int want = (2 * ctx->n_sm + units - 1) / units;        // about two CTAs per SM
+    int want;
+    if (resolve_kernel(s) == LVSPEC_KERNEL_TCGEN05)
+        want = ctx->n_sm / units;                          // one CTA per SM, one wave
+    else
+        want = (2 * ctx->n_sm + units - 1) / units;        // about two CTAs per SM
     if (want < 1) want = 1;
     if (want > tiles) want = tiles;
     if (want > 256) want = 256;
@@ -168,9 +179,14 @@ lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, con
     int launches = 0;
     cudaError_t e;
     const int kernel = resolve_kernel(s);
-    if (kernel == LVSPEC_KERNEL_TCGEN05)
-        return fail(ctx, LVSPEC_ERR_UNSUPPORTED, "tcgen05 kernel not built");
-    e = launch_attn_simt(p, seq, ctx->stream, &launches);
+    if (kernel == LVSPEC_KERNEL_TCGEN05) {
+        if (!attn_tc_supported(p))
+            return fail(ctx, LVSPEC_ERR_UNSUPPORTED,
+                        "the tcgen05 kernel needs head_dim 128 and kv_capacity >= 128");
+        e = launch_attn_tc(p, seq, ctx->stream, &launches);
+    } else {
+        e = launch_attn_simt(p, seq, ctx->stream, &launches);
+    }
     ctx->launches += launches;
     if (e != cudaSuccess) return cuda_fail(ctx, "attention kernel launch", e);
     launches = 0;

@@ -40,6 +40,9 @@ static inline size_t part_stat_elems(const AttnParams &p)
 
 cudaError_t launch_attn_simt(const AttnParams &p, const SeqInfo &seq, cudaStream_t stream,
                              int *launches);
+bool attn_tc_supported(const AttnParams &p);
+cudaError_t launch_attn_tc(const AttnParams &p, const SeqInfo &seq, cudaStream_t stream,
+                           int *launches);
 cudaError_t launch_attn_combine(const AttnParams &p, cudaStream_t stream, int *launches);
 
 struct AcceptParams {
