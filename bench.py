@@ -14,6 +14,7 @@ path; the value is the sum over ranks divided by the slowest rank's time.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -43,6 +44,9 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch layer by layer, no CUDA graph")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="override the config's layer count (a smaller case of the same kernel for "
+                         "profiler captures; the line then says so and is not a bench value)")
     return ap.parse_args()
 
 
@@ -154,13 +158,19 @@ def workload_desc(cfg, n_gpus):
                         f"KV {cfg.kv_len} ({cfg.span[1] - cfg.span[0]} visual), vocab {cfg.vocab}",
             "kv_bytes_per_step": cfg.kv_bytes_per_layer * cfg.layers,
             "l2": "inputs larger than L2 (every layer streams its own K/V cache)",
-            "parallelism": "replicas only" if n_gpus > 1 else "1 GPU"}
+            "parallelism": "replicas only" if n_gpus > 1 else "1 GPU",
+            "layers_overridden": cfg.layers != full_layers(cfg)}
+
+
+def full_layers(cfg):
+    from paper_2604_05650_b200 import workloads as W
+    return W.CONFIGS[cfg_id_of(cfg)].layers
 
 
 def cfg_id_of(cfg):
     from paper_2604_05650_b200 import workloads as W
     for i, c in W.CONFIGS.items():
-        if c is cfg:
+        if c.name == cfg.name:
             return i
     return -1
 
@@ -394,6 +404,8 @@ def main():
     args = parse()
     from paper_2604_05650_b200 import workloads as W
     cfg = W.CONFIGS[args.config]
+    if args.layers > 0:
+        cfg = dataclasses.replace(cfg, layers=args.layers)
     if args.impl == "reference":
         run_reference(args, cfg)
     else:
