@@ -220,6 +220,49 @@ lvspec_status_t lvspec_loose_accept_host(lvspec_ctx_t *ctx, int32_t batch, int32
                                          const lvspec_thresholds_t *thresholds,
                                          int32_t shift_window, int32_t *accept_len);
 
+/* ---- loose acceptance without any allocation ---------------------------------
+ *
+ * The paper has no counterpart of this call: it is the operation of
+ * lvspec_loose_accept, offered to callers that are not allowed to allocate
+ * device memory: an inference server whose own pool already owns the GPU's
+ * memory, a process that must stay inside a memory budget fixed at start-up, or
+ * a latency-critical loop that cannot afford the device-wide synchronisation a
+ * cudaMalloc or cudaFree may bring.  It takes no context.  Its scratch memory
+ * (argmax partials, per-sequence tickets, a status word: about 66 KB) is a
+ * fixed array inside the library's device image; every GPU on which the
+ * library's code is loaded holds that array until the process ends.
+ *
+ * Arguments, operation and results are those of lvspec_loose_accept, except:
+ *   - work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL =
+ *     the default stream) of the CALLER'S CURRENT DEVICE, and all pointers must
+ *     belong to that device;
+ *   - batch * gamma must not exceed LVSPEC_STATIC_MAX_ROWS; larger calls are
+ *     refused with LVSPEC_ERR_UNSUPPORTED and launch nothing;
+ *   - a NaN logit still ranks as -inf, but is not reported (there is no context
+ *     to read a status word from);
+ *   - `error_text` (host, may be NULL) receives a NUL-terminated description of
+ *     at most error_text_len bytes when the call fails, "" when it succeeds.
+ *
+ * The call itself never calls cudaMalloc, cudaFree or any allocating routine.
+ * The first call on each device looks up the device address of the array
+ * (cudaGetSymbolAddress); make that first call outside any stream capture.
+ * Later calls only enqueue two kernels (one clears the tickets).
+ *
+ * All calls on a device share the one array, and it keeps whatever the last
+ * call left in it; each call clears the part that has to start at zero.  Two
+ * calls whose kernels can overlap on the GPU (different streams, or several
+ * host threads without stream ordering between them) race on it and give
+ * wrong results: order them on one stream or with events. */
+#define LVSPEC_STATIC_MAX_ROWS  1024  /* batch * gamma */
+#define LVSPEC_STATIC_MAX_SLOTS 8192  /* argmax partials the array holds */
+lvspec_status_t lvspec_loose_accept_static(void *cuda_stream, int32_t batch, int32_t gamma,
+                                           int32_t vocab, int32_t n_mass_heads,
+                                           const float *target_logits,
+                                           const int32_t *draft_tokens, const float *visual_mass,
+                                           const lvspec_thresholds_t *thresholds,
+                                           int32_t shift_window, int32_t *accept_len,
+                                           char *error_text, size_t error_text_len);
+
 #ifdef __cplusplus
 }
 #endif

@@ -28,6 +28,7 @@ EXPORTS = (
     "lvspec_last_error", "lvspec_status_string", "lvspec_launch_count",
     "lvspec_attention_splits", "lvspec_verify_attention", "lvspec_verify_attention_host",
     "lvspec_loose_accept", "lvspec_loose_accept_ex", "lvspec_loose_accept_host",
+    "lvspec_loose_accept_static",
 )
 
 
@@ -81,6 +82,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lvspec_loose_accept.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp]
     lib.lvspec_loose_accept_ex.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp, vp, vp]
     lib.lvspec_loose_accept_host.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp]
+    lib.lvspec_loose_accept_static.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp,
+                                               ctypes.c_char_p, ctypes.c_size_t]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if fn.restype is ctypes.c_int and name not in ("lvspec_attention_splits",):
@@ -185,6 +188,28 @@ class Context:
             self._h, batch, gamma, vocab, n_mass_heads, _addr(target_logits),
             _addr(draft_tokens), _addr(visual_mass), ctypes.byref(th), int(shift_window),
             _addr(accept_len)))
+
+
+STATIC_MAX_ROWS = 1024
+
+
+def loose_accept_static(stream, batch, gamma, vocab, n_mass_heads, target_logits, draft_tokens,
+                        visual_mass, accept_len, shift_window, lam: float = 0.7,
+                        n_loose: int = -1) -> None:
+    """``lvspec_loose_accept_static``: the acceptance pass for callers that may
+    not allocate device memory.  No context; runs on the current CUDA device,
+    on ``stream`` (raw cudaStream_t address, an object with ``cuda_stream``, or
+    None).  Raises ``LvspecError`` with the library's own text on failure."""
+    lib = load_library()
+    s = getattr(stream, "cuda_stream", stream)
+    th = Thresholds(float(lam), int(n_loose), 0)
+    text = ctypes.create_string_buffer(256)
+    st = lib.lvspec_loose_accept_static(
+        ctypes.c_void_p(int(s) if s else 0), batch, gamma, vocab, n_mass_heads,
+        _addr(target_logits), _addr(draft_tokens), _addr(visual_mass), ctypes.byref(th),
+        int(shift_window), _addr(accept_len), text, len(text))
+    if st != OK:
+        raise LvspecError(st, text.value.decode())
 
 
 HAVE_TCGEN05 = True
