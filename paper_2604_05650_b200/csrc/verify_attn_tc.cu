@@ -7,21 +7,25 @@
 //     S^T[pos, n] = K_tile[pos, :] . Q[n, :]          (MMA M = 128 positions, N = rows)
 //     O^T[d, n]  += V_tile[:, d]^T . P^T[:, n]        (MMA M = 128 channels,  N = rows)
 //     L[0..1, n] += [1; in_span]   . P^T[:, n]        (MMA M = 64: row 0 = l, row 1 = l_vis)
-// so every TMEM lane of S^T is one cache position (all 128 softmax threads do
+// so every TMEM lane of S^T is one cache position (all softmax threads do
 // useful exponentials) and the padded dimension is N (granularity 16), not M.
 // The softmax denominators l and the visual-span numerators l_vis come out of
 // the tensor core as two extra accumulator rows fed by a constant 0/1 tile.
 //
-// The running maximum m[n] is kept fixed while scores stay within 2^60 of it:
-// the tile's own maximum (a cross-lane reduction in this layout) is only taken
-// when a score exceeds the guard, in which case the accumulators are rescaled.
-// fp32 and bf16 share the exponent range, so nothing is lost in between.
+// The reference exponent m[n] of a row is the score of the first position of
+// the split and stays fixed while scores stay within 2^60 of it; only when a
+// score runs past that guard is the tile's maximum taken (a cross-lane
+// reduction in this layout) and the accumulators rescaled.  fp32 and bf16
+// share the exponent range, so nothing is lost in between.
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM owner),
-// warps 2-3 = prologue helpers, warps 4-7 = softmax (TMEM lane quarter = warp
-// % 4).  K and V tiles sit in separate shared-memory rings, each slot two
-// 128-position x 64-channel boxes with the 128-byte swizzle.  Every mbarrier
-// wait is bounded; a wait that gives up raises LVSPEC_DEV_WAIT_EXPIRED.
+// Warp roles (320 threads): warp 0 = TMA producer, warp 1 = MMA issuer and
+// TMEM owner, warps 2-5 and 6-9 = two softmax groups.  Both groups work on
+// every tile, each on its own half of the N columns (TMEM lane quarter = warp
+// % 4), so the two halves never interact: each has its own m, its own guard
+// and its own rescale.  K and V tiles sit in separate shared-memory rings,
+// each slot two 128-position x 64-channel boxes with the 128-byte swizzle; Q
+// arrives by TMA in the same layout.  Every mbarrier wait is bounded; a wait
+// that gives up raises LVSPEC_DEV_WAIT_EXPIRED.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -34,7 +38,8 @@ namespace {
 using namespace ptx;
 
 constexpr int kTilePos = 128;
-constexpr int kThreads = 256;
+constexpr int kThreads = 320;
+constexpr int kSoftmaxWarp0 = 2;            // first softmax warp
 constexpr uint32_t kBoxBytes = 16384;       // 128 positions x 64 channels bf16
 constexpr uint32_t kSlotBytes = 2 * kBoxBytes;
 constexpr uint32_t kA2Bytes = 2048;         // one 64 x 16 constant tile
@@ -63,7 +68,7 @@ __host__ __device__ inline SmemMap smem_map(const TcConfig &c)
     s.m = o;    o += c.n_pad * 4;
     s.dl = o;   o += c.n_pad * 4;
     s.tmx = o;  o += 4 * c.n_pad * 4;
-    s.bars = o; o += 8 * (2 * c.ks + 2 * c.vs + 4 + 2 * c.pb + 1);
+    s.bars = o; o += 8 * (2 * c.ks + 2 * c.vs + 4 + 2 * c.pb + 3);
     s.misc = o; o += 16;
     s.total = o;
     return s;
@@ -76,16 +81,60 @@ struct TcParams {
 
 __device__ __forceinline__ bool wait_unconditional(uint32_t bar, uint32_t parity)
 {
-    // used only while tearing down after an abort: time-bounded, ignores the flag
+    // used while tearing down: time-bounded, ignores the abort flag
     const uint64_t t0 = global_timer_ns();
     while (!mbar_try_wait(bar, parity))
         if (global_timer_ns() - t0 > 1000000000ull) return false;
     return true;
 }
 
+// named barrier over the 128 threads of one softmax group (ids 1 and 2)
+__device__ __forceinline__ void group_sync(int id)
+{
+    asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory");
+}
+__device__ __forceinline__ bool group_any(int id, bool pred)
+{
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %2, 0;\n\t"
+        "bar.red.or.pred p, %1, 128, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"(id), "r"((uint32_t)pred)
+        : "memory");
+    return out != 0;
+}
+
+// exp2 of eight scaled scores of one position, packed to bf16; returns their maximum
+__device__ __forceinline__ float exp_chunk(const uint32_t (&r)[8], const float *m8, float scale,
+                                           bool tail, int col0, int G, int gmin, uint4 *dst)
+{
+    const float4 ma = *reinterpret_cast<const float4 *>(m8);
+    const float4 mb = *reinterpret_cast<const float4 *>(m8 + 4);
+    const float mm[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
+    float x[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) x[k] = fmaf(__uint_as_float(r[k]), scale, -mm[k]);
+    if (tail) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) x[k] = ((col0 + k) / G >= gmin) ? x[k] : -INFINITY;
+    }
+    float mx = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])),
+                     fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
+    uint4 pk;
+    pk.x = pack_bf16x2(ex2(x[0]), ex2(x[1]));
+    pk.y = pack_bf16x2(ex2(x[2]), ex2(x[3]));
+    pk.z = pack_bf16x2(ex2(x[4]), ex2(x[5]));
+    pk.w = pack_bf16x2(ex2(x[6]), ex2(x[7]));
+    *dst = pk;
+    return mx;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUtensorMap tmap_k,
-               const __grid_constant__ CUtensorMap tmap_v)
+               const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_q)
 {
     extern __shared__ uint8_t smem_raw[];
     const AttnParams &p = P.a;
@@ -96,15 +145,20 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     const int M = p.M, G = p.G, gamma = p.gamma, NP = cfg.n_pad;
     const int n8 = (M + 7) >> 3;
 
+    // tiles [t_begin, t_begin + T) of this split: equal shares, sizes differ by at most one
     const int n_tiles = (L + kTilePos - 1) / kTilePos;
-    const int tiles_per_split = (n_tiles + p.n_split - 1) / p.n_split;
-    const int t_begin = split * tiles_per_split;
-    const int T = min(n_tiles, t_begin + tiles_per_split) - t_begin;
+    const int t_begin = (int)(((long long)split * n_tiles) / p.n_split);
+    const int T = (int)(((long long)(split + 1) * n_tiles) / p.n_split) - t_begin;
 
     const size_t unit = ((size_t)b * p.Hkv + kvh) * p.n_split + split;
     float *part_o = p.part_o + unit * (size_t)M * 128;
     float *part_stat = p.part_stat + unit * (size_t)M * 4;
     if (T <= 0) {   // a split with no tile: contributes nothing
+        if (tid == 0) {
+            grid_dependency_wait();
+            grid_launch_dependents();
+        }
+        __syncthreads();
         for (int r = tid; r < M; r += kThreads)
             *reinterpret_cast<float4 *>(part_stat + r * 4) = make_float4(kMFloor, 0.f, 0.f, 0.f);
         return;
@@ -131,61 +185,98 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     auto p_full = [&](int s) { return bar1 + 8 * (4 + s); };
     auto p_free = [&](int s) { return bar1 + 8 * (4 + cfg.pb + s); };
     const uint32_t drain_bar = bar1 + 8 * (4 + 2 * cfg.pb);
+    const uint32_t done_bar = drain_bar + 8;
+    const uint32_t q_full = drain_bar + 16;
+    const int bh = b * p.Hkv + kvh;
+
+    auto load_k = [&](int i) {
+        const int ks = i % cfg.ks, pos0 = (t_begin + i) * kTilePos;
+        mbar_arrive_expect_tx(k_full(ks), kSlotBytes);
+        tma_load_3d(base + sm.k + ks * kSlotBytes, &tmap_k, k_full(ks), 0, pos0, bh);
+        tma_load_3d(base + sm.k + ks * kSlotBytes + kBoxBytes, &tmap_k, k_full(ks), 64, pos0, bh);
+    };
+    auto load_v = [&](int i) {
+        const int vsl = i % cfg.vs, pos0 = (t_begin + i) * kTilePos;
+        mbar_arrive_expect_tx(v_full(vsl), kSlotBytes);
+        tma_load_3d(base + sm.v + vsl * kSlotBytes, &tmap_v, v_full(vsl), 0, pos0, bh);
+        tma_load_3d(base + sm.v + vsl * kSlotBytes + kBoxBytes, &tmap_v, v_full(vsl), 64, pos0, bh);
+    };
 
     // ------------------------------------------------------------------ prologue
-    if (tid == 0) {
-        for (int s = 0; s < cfg.ks; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); }
-        for (int s = 0; s < cfg.vs; ++s) { mbar_init(v_full(s), 1); mbar_init(v_empty(s), 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(s_full(s), 1); mbar_init(s_free(s), 128); }
-        for (int s = 0; s < cfg.pb; ++s) { mbar_init(p_full(s), 128); mbar_init(p_free(s), 1); }
-        mbar_init(drain_bar, 1);
-        *abort_flag = 0;
-        mbar_fence_init();
-        prefetch_tensormap(&tmap_k);
-        prefetch_tensormap(&tmap_v);
-    }
-    if (warp == 1) {
+    // The producer thread sets the barriers up and starts the first loads at
+    // once; the other warps prepare shared memory and TMEM meanwhile.
+    int first_k = 0, first_v = 0;   // loads issued before the CTA-wide barrier
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int s = 0; s < cfg.ks; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); }
+            for (int s = 0; s < cfg.vs; ++s) { mbar_init(v_full(s), 1); mbar_init(v_empty(s), 1); }
+            for (int s = 0; s < 2; ++s) { mbar_init(s_full(s), 1); mbar_init(s_free(s), 8); }
+            for (int s = 0; s < cfg.pb; ++s) { mbar_init(p_full(s), 8); mbar_init(p_free(s), 1); }
+            mbar_init(drain_bar, 1);
+            mbar_init(done_bar, 8);
+            mbar_init(q_full, 1);
+            *abort_flag = 0;
+            mbar_fence_init();
+            fence_proxy_async_smem();
+            // inputs may come from the kernel before this one in the stream
+            grid_dependency_wait();
+            mbar_arrive_expect_tx(q_full, (uint32_t)M * 256u);
+            tma_load_4d(base + sm.q, &tmap_q, q_full, 0, kvh * G, 0, b);
+            tma_load_4d(base + sm.q + NP * 128, &tmap_q, q_full, 64, kvh * G, 0, b);
+            first_k = min(T, cfg.ks);
+            first_v = min(T, cfg.vs);
+            for (int i = 0; i < first_v; ++i) {
+                if (i < first_k) load_k(i);
+                load_v(i);
+            }
+            grid_launch_dependents();
+        }
+        __syncwarp();
+    } else if (warp == 1) {
         tmem_alloc(base + sm.misc, (uint32_t)cfg.tmem_cols);
         tmem_relinquish();
-    }
-    if (warp == 2 || warp == 3) {
-        const int idx = tid - 64;
-        // Q rows of this KV head, K-major with the 128-byte swizzle: two halves of
-        // 64 channels, rows of 128 bytes, 16-byte chunk c of row r stored at c ^ (r % 8)
-        for (int i = idx; i < NP * 16; i += 64) {
-            const int r = i >> 4, c = i & 15, h = c >> 3, cc = c & 7;
-            uint4 val = make_uint4(0, 0, 0, 0);
-            if (r < M) {
-                const int g = r / G, hg = r - g * G;
-                const size_t off = (((size_t)b * gamma + g) * p.Hq + kvh * G + hg) * 128 + c * 8;
-                val = *reinterpret_cast<const uint4 *>(p.q + off);
-            }
-            uint8_t *dst = gbase + sm.q + h * (NP * 128) + (r >> 3) * 1024 + (r & 7) * 128 +
-                           ((cc ^ (r & 7)) << 4);
-            *reinterpret_cast<uint4 *>(dst) = val;
+    } else {
+        const int idx = tid - 64;   // 0..255
+        // rows M..NP-1 of Q are padding: zero them (the TMA boxes cover rows < M only)
+        for (int i = idx; i < (NP - M) * 16; i += 256) {
+            const int r = M + (i >> 4), c = i & 15, h = c >> 3, cc = c & 7;
+            *reinterpret_cast<uint4 *>(gbase + sm.q + h * (NP * 128) + r * 128 + cc * 16) =
+                make_uint4(0, 0, 0, 0);
         }
-        // P buffers and the constant tiles start as zeros
-        for (uint32_t i = idx * 16; i < (uint32_t)(cfg.pb * NP * 256) + 4 * kA2Bytes; i += 64 * 16)
+        // P buffers start as zeros (columns beyond the last chunk stay zero)
+        for (uint32_t i = idx * 16; i < (uint32_t)(cfg.pb * NP * 256); i += 256 * 16)
             *reinterpret_cast<uint4 *>(gbase + sm.p + i) = make_uint4(0, 0, 0, 0);
-        for (int n = idx; n < NP; n += 64) m_s[n] = kMFloor;
-        asm volatile("bar.sync 2, 64;" ::: "memory");
-        // constant 64 x 16 tiles (K-major, no swizzle: chunk c of 8 positions at
-        // c * 1024, row r at (r / 8) * 128 + (r % 8) * 16).  Row 0 = ones (sums l),
-        // row 1 = 1 inside the visual span (sums l_vis).
-        // tile 0: inside the span, 1: outside, 2: the 16-block holding span start,
-        // 3: the 16-block holding span end
-        if (idx < 64) {
-            const int tile = idx >> 4, kpos = idx & 15, c = kpos >> 3, e = kpos & 7;
-            uint16_t *t16 = reinterpret_cast<uint16_t *>(gbase + sm.a2 + tile * kA2Bytes + c * 1024);
-            int ind;
-            if (tile == 0) ind = 1;
-            else if (tile == 1) ind = 0;
-            else {
-                const int pos = ((tile == 2 ? vs : ve) & ~15) + kpos;
-                ind = (pos >= vs && pos < ve) ? 1 : 0;
+        for (int n = idx; n < NP; n += 256) m_s[n] = 0.f;
+        // constant 64 x 16 tiles (K-major, no swizzle: the 8 positions of chunk c
+        // at c * 1024, row r at (r / 8) * 128 + (r % 8) * 16).  Row 0 = ones (sums
+        // l), row 1 = 1 inside the visual span (sums l_vis), rows 2.. = 0.
+        // tile 0: block inside the span, 1: outside, 2: the 16-block holding the
+        // span start, 3: the 16-block holding the span end
+        for (uint32_t i = idx * 16; i < 4 * kA2Bytes; i += 256 * 16) {
+            const int tile = i / kA2Bytes, off = i % kA2Bytes;
+            const int c = off / 1024, rr = (off % 1024) / 16;   // rr = row index 0..63
+            uint4 val = make_uint4(0, 0, 0, 0);
+            if (rr < 2) {
+                uint16_t e[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    int ind = 1;
+                    if (rr == 1) {
+                        if (tile == 0) ind = 1;
+                        else if (tile == 1) ind = 0;
+                        else {
+                            const int pos = ((tile == 2 ? vs : ve) & ~15) + c * 8 + k;
+                            ind = (pos >= vs && pos < ve) ? 1 : 0;
+                        }
+                    }
+                    e[k] = ind ? 0x3F80 : 0;
+                }
+                val.x = e[0] | ((uint32_t)e[1] << 16);
+                val.y = e[2] | ((uint32_t)e[3] << 16);
+                val.z = e[4] | ((uint32_t)e[5] << 16);
+                val.w = e[6] | ((uint32_t)e[7] << 16);
             }
-            t16[e] = 0x3F80;                    // row 0
-            t16[8 + e] = ind ? 0x3F80 : 0;      // row 1
+            *reinterpret_cast<uint4 *>(gbase + sm.a2 + i) = val;
         }
         fence_proxy_async_smem();
     }
@@ -194,34 +285,29 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tm_s0 = tmem_base, tm_o = tmem_base + 2 * NP, tm_l = tmem_base + 3 * NP;
-    const int bh = b * p.Hkv + kvh;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            int i = 0;
-            for (; i < T; ++i) {
-                const int pos0 = (t_begin + i) * kTilePos;
-                const int ks = i % cfg.ks;
-                if (i >= cfg.ks && !mbar_wait(k_empty(ks), ((i / cfg.ks) - 1) & 1, abort_flag)) break;
-                mbar_arrive_expect_tx(k_full(ks), kSlotBytes);
-                tma_load_3d(base + sm.k + ks * kSlotBytes, &tmap_k, k_full(ks), 0, pos0, bh);
-                tma_load_3d(base + sm.k + ks * kSlotBytes + kBoxBytes, &tmap_k, k_full(ks), 64, pos0, bh);
-                const int vsl = i % cfg.vs;
-                if (i >= cfg.vs && !mbar_wait(v_empty(vsl), ((i / cfg.vs) - 1) & 1, abort_flag)) {
-                    // the K load of this tile is already in flight: wait for it here
-                    wait_unconditional(k_full(ks), (i / cfg.ks) & 1);
-                    break;
+            int nk = first_k, nv = first_v;   // loads issued so far
+            while (nk < T || nv < T) {
+                if (nk < T) {
+                    if (!mbar_wait(k_empty(nk % cfg.ks), ((nk / cfg.ks) - 1) & 1, abort_flag)) break;
+                    load_k(nk);
+                    ++nk;
                 }
-                mbar_arrive_expect_tx(v_full(vsl), kSlotBytes);
-                tma_load_3d(base + sm.v + vsl * kSlotBytes, &tmap_v, v_full(vsl), 0, pos0, bh);
-                tma_load_3d(base + sm.v + vsl * kSlotBytes + kBoxBytes, &tmap_v, v_full(vsl), 64, pos0, bh);
+                if (nv < T) {
+                    if (!mbar_wait(v_empty(nv % cfg.vs), ((nv / cfg.vs) - 1) & 1, abort_flag)) break;
+                    load_v(nv);
+                    ++nv;
+                }
             }
             if (*abort_flag) {
                 // wait (bounded) for the copies still in flight before the CTA leaves
-                for (int j = max(0, i - cfg.ks); j < i; ++j)
+                wait_unconditional(q_full, 0);
+                for (int j = max(0, nk - cfg.ks); j < nk; ++j)
                     wait_unconditional(k_full(j % cfg.ks), (j / cfg.ks) & 1);
-                for (int j = max(0, i - cfg.vs); j < i; ++j)
+                for (int j = max(0, nv - cfg.vs); j < nv; ++j)
                     wait_unconditional(v_full(j % cfg.vs), (j / cfg.vs) & 1);
             }
         }
@@ -231,53 +317,74 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             const uint32_t idesc_qk = make_idesc_bf16(128, NP, 0, 0);
             const uint32_t idesc_pv = make_idesc_bf16(128, NP, 1, 1);
             const uint32_t idesc_sum = make_idesc_bf16(64, NP, 0, 1);
+            // descriptors: everything but the start address is fixed, and the start
+            // address field (address / 16) moves by compile-time steps
+            const uint64_t kd0 = make_smem_desc(base + sm.k, 16, 1024, kSwizzle128B);
+            const uint64_t vd0 = make_smem_desc(base + sm.v, kBoxBytes, 1024, kSwizzle128B);
+            const uint64_t pd0 = make_smem_desc(base + sm.p, 128, 2048, kSwizzleNone);
+            const uint64_t a2d0 = make_smem_desc(base + sm.a2, 1024, 128, kSwizzleNone);
+            uint64_t qd[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                qd[j] = make_smem_desc(base + sm.q + (j >> 2) * (NP * 128) + (j & 3) * 32, 16, 1024,
+                                       kSwizzle128B);
             auto issue_qk = [&](int i) -> bool {
                 const int ks = i % cfg.ks, sb = i & 1;
                 if (!mbar_wait(k_full(ks), (i / cfg.ks) & 1, abort_flag)) return false;
                 if (i >= 2 && !mbar_wait(s_free(sb), ((i >> 1) - 1) & 1, abort_flag)) return false;
                 tc_fence_after();
-                const uint32_t kslot = base + sm.k + ks * kSlotBytes;
+                const uint64_t kd = kd0 + (uint64_t)(ks * (kSlotBytes >> 4));
+                const uint32_t d = tm_s0 + sb * NP;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const uint64_t da = make_smem_desc(kslot + (j >> 2) * kBoxBytes + (j & 3) * 32, 16,
-                                                       1024, kSwizzle128B);
-                    const uint64_t db = make_smem_desc(base + sm.q + (j >> 2) * (NP * 128) + (j & 3) * 32,
-                                                       16, 1024, kSwizzle128B);
-                    mma_f16_ss(tm_s0 + sb * NP, da, db, idesc_qk, j > 0);
-                }
+                for (int j = 0; j < 8; ++j)
+                    mma_f16_ss(d, kd + (uint64_t)((j >> 2) * (kBoxBytes >> 4) + (j & 3) * 2), qd[j],
+                               idesc_qk, j > 0);
                 mma_commit(s_full(sb));
                 mma_commit(k_empty(ks));
                 return true;
             };
-            bool ok = issue_qk(0);
+            bool ok = mbar_wait(q_full, 0, abort_flag) && issue_qk(0);
             for (int i = 0; ok && i < T; ++i) {
                 if (i + 1 < T && !issue_qk(i + 1)) break;
                 const int pb = i % cfg.pb, vsl = i % cfg.vs;
                 if (!mbar_wait(p_full(pb), (i / cfg.pb) & 1, abort_flag)) break;
                 if (!mbar_wait(v_full(vsl), (i / cfg.vs) & 1, abort_flag)) break;
                 tc_fence_after();
-                const uint32_t vslot = base + sm.v + vsl * kSlotBytes;
-                const uint32_t pbuf = base + sm.p + pb * (NP * 256);
+                // V^T: channels contiguous (M-major), 64-channel halves kBoxBytes apart,
+                // groups of 8 positions 1024 bytes apart.  P^T: rows contiguous in
+                // 16-byte chunks (N-major), chunk stride 2048, groups of 8 positions 128
+                // bytes apart.
+                const uint64_t vd = vd0 + (uint64_t)(vsl * (kSlotBytes >> 4));
+                const uint64_t pd = pd0 + (uint64_t)(pb * ((NP * 256) >> 4));
                 const int pos0 = (t_begin + i) * kTilePos;
+                // constant tile per block of 16 positions: 0 inside the span, 1 outside,
+                // 2 / 3 the blocks holding the span's start / end
+                int uniform = -1;
+                if (pos0 >= vs && pos0 + kTilePos <= ve) uniform = 0;
+                else if (pos0 + kTilePos <= vs || pos0 >= ve) uniform = 1;
+                const uint32_t first_acc = i > 0 ? 1u : 0u;
+                if (uniform >= 0) {
+                    const uint64_t d2 = a2d0 + (uint64_t)(uniform * (kA2Bytes >> 4));
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    // V^T: channels contiguous (M-major), 64-channel halves kBoxBytes apart,
-                    // groups of 8 positions 1024 bytes apart
-                    const uint64_t da = make_smem_desc(vslot + j * 2048, kBoxBytes, 1024, kSwizzle128B);
-                    // P^T: rows contiguous in 16-byte chunks (N-major), chunk stride 2048,
-                    // groups of 8 positions 128 bytes apart
-                    const uint64_t db = make_smem_desc(pbuf + j * 256, 128, 2048, kSwizzleNone);
-                    const uint32_t acc = (i > 0 || j > 0) ? 1u : 0u;
-                    mma_f16_ss(tm_o, da, db, idesc_pv, acc);
-                    const int pblk = pos0 + 16 * j;
-                    int tile;
-                    if (pblk >= vs && pblk + 16 <= ve) tile = 0;
-                    else if (pblk + 16 <= vs || pblk >= ve) tile = 1;
-                    else if ((vs & ~15) == pblk) tile = 2;
-                    else tile = 3;
-                    const uint64_t d2 = make_smem_desc(base + sm.a2 + tile * kA2Bytes, 1024, 128,
-                                                       kSwizzleNone);
-                    mma_f16_ss(tm_l, d2, db, idesc_sum, acc);
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t acc = j > 0 ? 1u : first_acc;
+                        mma_f16_ss(tm_o, vd + (uint64_t)(j * 128), pd + (uint64_t)(j * 16), idesc_pv, acc);
+                        mma_f16_ss(tm_l, d2, pd + (uint64_t)(j * 16), idesc_sum, acc);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t acc = j > 0 ? 1u : first_acc;
+                        const int pblk = pos0 + 16 * j;
+                        int tile;
+                        if (pblk >= vs && pblk + 16 <= ve) tile = 0;
+                        else if (pblk + 16 <= vs || pblk >= ve) tile = 1;
+                        else if ((vs & ~15) == pblk) tile = 2;
+                        else tile = 3;
+                        mma_f16_ss(tm_o, vd + (uint64_t)(j * 128), pd + (uint64_t)(j * 16), idesc_pv, acc);
+                        mma_f16_ss(tm_l, a2d0 + (uint64_t)(tile * (kA2Bytes >> 4)),
+                                   pd + (uint64_t)(j * 16), idesc_sum, acc);
+                    }
                 }
                 mma_commit(v_empty(vsl));
                 mma_commit(p_free(pb));
@@ -286,12 +393,16 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             mma_commit(drain_bar);
             wait_unconditional(drain_bar, 0);
         }
-    } else if (warp >= 4) {
+    } else {
         // ------------------------------------------------------------ softmax warps
-        const int wq = warp & 3;
+        const int grp = (warp - kSoftmaxWarp0) >> 2;    // column half this warp works on
+        const int bar_id = 1 + grp;
+        const int wq = warp & 3;                        // TMEM lane quarter of this warp
         const int row = wq * 32 + lane;                 // TMEM lane = position inside the tile
+        const int gtid = ((warp - kSoftmaxWarp0) & 3) * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
-        const int wtid = tid - 128;
+        const int n_a = (n8 + 1) >> 1;
+        const int c_lo = grp ? n_a : 0, c_hi = grp ? n8 : n_a;   // chunks of 8 columns
         const float scale = p.scale_log2;
         for (int i = 0; i < T; ++i) {
             const int pos0 = (t_begin + i) * kTilePos;
@@ -299,10 +410,25 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             const int sb = i & 1, pb = i % cfg.pb;
             mbar_wait(s_full(sb), (i >> 1) & 1, abort_flag);
             tc_fence_after();
-            if (i >= cfg.pb) mbar_wait(p_free(pb), ((i / cfg.pb) - 1) & 1, abort_flag);
+            const uint32_t s_addr = tm_s0 + sb * NP + lane_addr;
+            if (i == 0) {
+                // reference exponent of each row: its score at the split's first position
+                if (wq == 0) {
+                    for (int c8 = c_lo; c8 < c_hi; ++c8) {
+                        uint32_t r[8];
+                        tmem_ld_x8(s_addr + c8 * 8, r);
+                        tmem_wait_ld();
+                        if (lane == 0) {
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) m_s[c8 * 8 + k] = __uint_as_float(r[k]) * scale;
+                        }
+                    }
+                }
+                group_sync(bar_id);
+            }
             const bool tail = pos0 + kTilePos > L - gamma;
             const int gmin = pos - L + gamma;           // queries g < gmin do not see `pos`
-            if (tail) {
+            if (tail && grp == 0) {
                 // slots at or beyond kv_len hold whatever the cache holds: zero their V
                 // rows so that 0 * junk cannot poison the accumulators
                 mbar_wait(v_full(i % cfg.vs), (i / cfg.vs) & 1, abort_flag);
@@ -315,39 +441,27 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                     }
                 }
             }
+            if (i >= cfg.pb) mbar_wait(p_free(pb), ((i / cfg.pb) - 1) & 1, abort_flag);
             uint8_t *prow = gbase + sm.p + pb * (NP * 256) + row * 16;
-            const uint32_t s_addr = tm_s0 + sb * NP + lane_addr;
 
             for (int attempt = 0; attempt < 3; ++attempt) {
                 float gmax = -INFINITY;
-                for (int c8 = 0; c8 < n8; ++c8) {
-                    uint32_t r[8];
-                    tmem_ld_x8(s_addr + c8 * 8, r);
-                    const float4 ma = *reinterpret_cast<const float4 *>(m_s + c8 * 8);
-                    const float4 mb = *reinterpret_cast<const float4 *>(m_s + c8 * 8 + 4);
-                    const float mm[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
+                for (int c8 = c_lo; c8 < c_hi; c8 += 2) {
+                    uint32_t r0[8], r1[8];
+                    const bool two = c8 + 1 < c_hi;
+                    tmem_ld_x8(s_addr + c8 * 8, r0);
+                    if (two) tmem_ld_x8(s_addr + c8 * 8 + 8, r1);
                     tmem_wait_ld();
-                    float x[8];
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) x[k] = fmaf(__uint_as_float(r[k]), scale, -mm[k]);
-                    if (tail) {
-#pragma unroll
-                        for (int k = 0; k < 8; ++k)
-                            x[k] = ((c8 * 8 + k) / G >= gmin) ? x[k] : -INFINITY;
-                    }
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) gmax = fmaxf(gmax, x[k]);
-                    uint4 pk;
-                    pk.x = pack_bf16x2(ex2(x[0]), ex2(x[1]));
-                    pk.y = pack_bf16x2(ex2(x[2]), ex2(x[3]));
-                    pk.z = pack_bf16x2(ex2(x[4]), ex2(x[5]));
-                    pk.w = pack_bf16x2(ex2(x[6]), ex2(x[7]));
-                    *reinterpret_cast<uint4 *>(prow + c8 * 2048) = pk;
+                    gmax = fmaxf(gmax, exp_chunk(r0, m_s + c8 * 8, scale, tail, c8 * 8, G, gmin,
+                                                 reinterpret_cast<uint4 *>(prow + c8 * 2048)));
+                    if (two)
+                        gmax = fmaxf(gmax, exp_chunk(r1, m_s + c8 * 8 + 8, scale, tail, c8 * 8 + 8, G, gmin,
+                                                     reinterpret_cast<uint4 *>(prow + (c8 + 1) * 2048)));
                 }
-                if (!wg_any(gmax > kGuard)) break;
+                if (!group_any(bar_id, gmax > kGuard)) break;
 
                 // ---- a score ran past the guard: move m up to the tile maximum ----
-                for (int c8 = 0; c8 < n8; ++c8) {
+                for (int c8 = c_lo; c8 < c_hi; ++c8) {
                     uint32_t r[8];
                     tmem_ld_x8(s_addr + c8 * 8, r);
                     tmem_wait_ld();
@@ -361,8 +475,8 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                         if (lane == 0) tmx_s[wq * NP + c8 * 8 + k] = s2;
                     }
                 }
-                wg_sync();
-                for (int n = wtid; n < n8 * 8; n += 128) {
+                group_sync(bar_id);
+                for (int n = c_lo * 8 + gtid; n < c_hi * 8; n += 128) {
                     const float mt = fmaxf(fmaxf(tmx_s[n], tmx_s[NP + n]),
                                            fmaxf(tmx_s[2 * NP + n], tmx_s[3 * NP + n]));
                     const float mo = m_s[n];
@@ -370,13 +484,13 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                     dl_s[n] = mo - mn;              // <= 0
                     m_s[n] = mn;
                 }
-                wg_sync();
+                group_sync(bar_id);
                 if (i > 0) {
-                    // O^T and the sums were accumulated under the old m: rescale them
-                    // once PV(i-1) has finished
+                    // O^T and the sums were accumulated under the old m: rescale this
+                    // group's columns once PV(i-1) has finished
                     mbar_wait(p_free((i - 1) % cfg.pb), ((i - 1) / cfg.pb) & 1, abort_flag);
                     tc_fence_after();
-                    for (int c8 = 0; c8 < n8; ++c8) {
+                    for (int c8 = c_lo; c8 < c_hi; ++c8) {
                         uint32_t r[8];
                         tmem_ld_x8(tm_o + lane_addr + c8 * 8, r);
                         tmem_wait_ld();
@@ -396,20 +510,23 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                     tmem_wait_st();
                     tc_fence_before();
                 }
-                wg_sync();
+                group_sync(bar_id);
             }
-            // S^T has been read: the MMA warp may overwrite this buffer
+            // S^T has been read and P^T (with any zeroed V rows) is in shared memory:
+            // one arrival per warp tells the MMA warp
             tc_fence_before();
-            mbar_arrive(s_free(sb));
-            // P^T (and zeroed V rows) are in shared memory: visible to the tensor core
             fence_proxy_async_smem();
-            mbar_arrive(p_full(pb));
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(s_free(sb));
+                mbar_arrive(p_full(pb));
+            }
         }
 
         // ---------------------------------------------------------------- epilogue
         mbar_wait(p_free((T - 1) % cfg.pb), ((T - 1) / cfg.pb) & 1, abort_flag);
         tc_fence_after();
-        for (int c8 = 0; c8 < n8; ++c8) {
+        for (int c8 = c_lo; c8 < c_hi; ++c8) {
             uint32_t r[8];
             tmem_ld_x8(tm_o + lane_addr + c8 * 8, r);
             tmem_wait_ld();
@@ -432,12 +549,19 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             }
         }
         tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(done_bar);
     }
 
     // ------------------------------------------------------------------ teardown
-    __syncthreads();
-    if (tid == 0 && *abort_flag) atomicOr(p.status, LVSPEC_DEV_WAIT_EXPIRED);
+    // TMEM goes back once the MMAs have drained and every softmax warp is done
     if (warp == 1) {
+        if (lane == 0) {
+            bool all_done = false;
+            for (int tries = 0; tries < 4 && !all_done; ++tries) all_done = wait_unconditional(done_bar, 0);
+            if (*abort_flag || !all_done) atomicOr(p.status, LVSPEC_DEV_WAIT_EXPIRED);
+        }
+        __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, (uint32_t)cfg.tmem_cols);
     }
@@ -476,13 +600,33 @@ bool make_kv_map(CUtensorMap *map, const void *ptr, int Lmax, int BH)
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// q [B][gamma][Hq][128] bf16 as a 4-D tensor; one box = 64 channels of the G heads of one
+// KV head for all gamma queries: its rows land in shared memory in the order g * G + hg
+bool make_q_map(CUtensorMap *map, const void *ptr, int B, int gamma, int Hq, int G)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {128, (cuuint64_t)Hq, (cuuint64_t)gamma, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {256, (cuuint64_t)Hq * 256, (cuuint64_t)gamma * Hq * 256};
+    const cuuint32_t box[4] = {64, (cuuint32_t)G, (cuuint32_t)gamma, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(ptr), dims, strides, box,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr uint32_t kMaxSmem = 232448 - 1024;   // 227 KB less the alignment slack
+
 TcConfig pick_config(int M)
 {
     TcConfig c;
     c.n_pad = (M + 15) & ~15;
-    if (c.n_pad <= 64) { c.ks = 2; c.vs = 3; c.pb = 2; }
-    else if (c.n_pad <= 96) { c.ks = 2; c.vs = 2; c.pb = 2; }
-    else { c.ks = 2; c.vs = 2; c.pb = 1; }
+    // deepest K/V rings that fit, two P buffers before a third V slot is given up
+    const int tries[4][3] = {{2, 3, 2}, {2, 3, 1}, {2, 2, 2}, {2, 2, 1}};
+    for (int t = 0; t < 4; ++t) {
+        c.ks = tries[t][0]; c.vs = tries[t][1]; c.pb = tries[t][2];
+        if (smem_map(c).total <= kMaxSmem) break;
+    }
     int cols = 32;
     while (cols < 4 * c.n_pad) cols <<= 1;
     c.tmem_cols = cols;
@@ -501,15 +645,16 @@ cudaError_t launch_attn_tc(const AttnParams &p, const SeqInfo &seq, cudaStream_t
     TcParams P;
     P.a = p;
     P.cfg = pick_config(p.M);
-    CUtensorMap mk, mv;
-    if (!make_kv_map(&mk, p.k, p.Lmax, p.B * p.Hkv) || !make_kv_map(&mv, p.v, p.Lmax, p.B * p.Hkv))
+    CUtensorMap mk, mv, mq;
+    if (!make_kv_map(&mk, p.k, p.Lmax, p.B * p.Hkv) || !make_kv_map(&mv, p.v, p.Lmax, p.B * p.Hkv) ||
+        !make_q_map(&mq, p.q, p.B, p.gamma, p.Hq, p.G))
         return cudaErrorInvalidValue;
     const size_t smem = smem_map(P.cfg).total + 1024;
     cudaError_t err = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)smem);
     if (err != cudaSuccess) return err;
     dim3 grid(p.n_split, p.Hkv, p.B);
-    attn_tc_kernel<<<grid, kThreads, smem, stream>>>(P, seq, mk, mv);
+    attn_tc_kernel<<<grid, kThreads, smem, stream>>>(P, seq, mk, mv, mq);
     ++*launches;
     return cudaGetLastError();
 }
