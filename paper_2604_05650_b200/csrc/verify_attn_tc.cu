@@ -18,8 +18,10 @@
 // reduction in this layout) and the accumulators rescaled.  fp32 and bf16
 // share the exponent range, so nothing is lost in between.
 //
-// Warp roles (320 threads): warp 0 = TMA producer, warp 1 = MMA issuer and
-// TMEM owner, warps 2-5 and 6-9 = two softmax groups.  Both groups work on
+// Warp roles (352 threads): warp 0 = TMA producer, warp 1 = issuer of the
+// K.Q^T MMAs and TMEM owner, warp 10 = issuer of the P.V and sum MMAs (one
+// thread each; two issuers because a single thread's issue rate, not the tensor
+// pipe, bounded the loop), warps 2-5 and 6-9 = two softmax groups.  Both groups work on
 // every tile, each on its own half of the N columns (TMEM lane quarter = warp
 // % 4), so the two halves never interact: each has its own m, its own guard
 // and its own rescale.  K and V tiles sit in separate shared-memory rings,
@@ -38,7 +40,8 @@ namespace {
 using namespace ptx;
 
 constexpr int kTilePos = 128;
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;
+constexpr int kPvWarp = 10;                 // issues the P.V and sum MMAs
 constexpr int kSoftmaxWarp0 = 2;            // first softmax warp
 constexpr uint32_t kBoxBytes = 16384;       // 128 positions x 64 channels bf16
 constexpr uint32_t kSlotBytes = 2 * kBoxBytes;
@@ -213,7 +216,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             for (int s = 0; s < 2; ++s) { mbar_init(s_full(s), 1); mbar_init(s_free(s), 8); }
             for (int s = 0; s < cfg.pb; ++s) { mbar_init(p_full(s), 8); mbar_init(p_free(s), 1); }
             mbar_init(drain_bar, 1);
-            mbar_init(done_bar, 8);
+            mbar_init(done_bar, 9);
             mbar_init(q_full, 1);
             *abort_flag = 0;
             mbar_fence_init();
@@ -235,7 +238,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     } else if (warp == 1) {
         tmem_alloc(base + sm.misc, (uint32_t)cfg.tmem_cols);
         tmem_relinquish();
-    } else {
+    } else if (warp < kPvWarp) {
         const int idx = tid - 64;   // 0..255
         // rows M..NP-1 of Q are padding: zero them (the TMA boxes cover rows < M only)
         for (int i = idx; i < (NP - M) * 16; i += 256) {
@@ -315,14 +318,9 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         // -------------------------------------------------------------- MMA issuer
         if (lane == 0) {
             const uint32_t idesc_qk = make_idesc_bf16(128, NP, 0, 0);
-            const uint32_t idesc_pv = make_idesc_bf16(128, NP, 1, 1);
-            const uint32_t idesc_sum = make_idesc_bf16(64, NP, 0, 1);
             // descriptors: everything but the start address is fixed, and the start
             // address field (address / 16) moves by compile-time steps
             const uint64_t kd0 = make_smem_desc(base + sm.k, 16, 1024, kSwizzle128B);
-            const uint64_t vd0 = make_smem_desc(base + sm.v, kBoxBytes, 1024, kSwizzle128B);
-            const uint64_t pd0 = make_smem_desc(base + sm.p, 128, 2048, kSwizzleNone);
-            const uint64_t a2d0 = make_smem_desc(base + sm.a2, 1024, 128, kSwizzleNone);
             uint64_t qd[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j)
@@ -343,9 +341,21 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 mma_commit(k_empty(ks));
                 return true;
             };
-            bool ok = mbar_wait(q_full, 0, abort_flag) && issue_qk(0);
-            for (int i = 0; ok && i < T; ++i) {
-                if (i + 1 < T && !issue_qk(i + 1)) break;
+            bool ok = mbar_wait(q_full, 0, abort_flag);
+            for (int i = 0; ok && i < T; ++i) ok = issue_qk(i);
+            // every MMA issued by this thread has finished before TMEM is released
+            mma_commit(drain_bar);
+            wait_unconditional(drain_bar, 0);
+        }
+    } else if (warp == kPvWarp) {
+        // ------------------------------------------------- P.V and sum MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc_pv = make_idesc_bf16(128, NP, 1, 1);
+            const uint32_t idesc_sum = make_idesc_bf16(64, NP, 0, 1);
+            const uint64_t vd0 = make_smem_desc(base + sm.v, kBoxBytes, 1024, kSwizzle128B);
+            const uint64_t pd0 = make_smem_desc(base + sm.p, 128, 2048, kSwizzleNone);
+            const uint64_t a2d0 = make_smem_desc(base + sm.a2, 1024, 128, kSwizzleNone);
+            for (int i = 0; i < T; ++i) {
                 const int pb = i % cfg.pb, vsl = i % cfg.vs;
                 if (!mbar_wait(p_full(pb), (i / cfg.pb) & 1, abort_flag)) break;
                 if (!mbar_wait(v_full(vsl), (i / cfg.vs) & 1, abort_flag)) break;
@@ -389,9 +399,8 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 mma_commit(v_empty(vsl));
                 mma_commit(p_free(pb));
             }
-            // every MMA issued by this thread has finished before TMEM is released
-            mma_commit(drain_bar);
-            wait_unconditional(drain_bar, 0);
+            // this thread's MMAs have finished: tell the TMEM owner
+            mma_commit(done_bar);
         }
     } else {
         // ------------------------------------------------------------ softmax warps
