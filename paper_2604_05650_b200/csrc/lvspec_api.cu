@@ -3,6 +3,7 @@
 // in the kernels; nothing here computes on the CPU.
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -22,6 +23,7 @@ struct lvspec_ctx {
     void *staging = nullptr;          // device copies for the *_host calls
     size_t staging_bytes = 0;
     uint64_t launches = 0;
+    bool pdl = true;                  // programmatic dependent launch between the attention kernels
     std::string error;
 };
 
@@ -168,6 +170,7 @@ lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, con
     p.M = p.gamma * p.G;
     p.n_split = s->n_split > 0 ? s->n_split : choose_splits(ctx, s, max_len);
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)p.D));
+    p.pdl = ctx->pdl ? 1 : 0;
 
     const size_t o_bytes = part_o_elems(p) * sizeof(float);
     const size_t st_bytes = part_stat_elems(p) * sizeof(float);
@@ -311,6 +314,7 @@ lvspec_status_t lvspec_create(lvspec_ctx_t **out, int device)
         return LVSPEC_ERR_UNSUPPORTED;
     }
     ctx->n_sm = prop.multiProcessorCount;
+    if (const char *e = std::getenv("LVSPEC_NO_PDL")) ctx->pdl = !(e[0] && e[0] != '0');
     const size_t small = sizeof(uint32_t) * (1 + LVSPEC_MAX_BATCH);
     if ((e = cudaMalloc(reinterpret_cast<void **>(&ctx->status), small)) != cudaSuccess ||
         (e = cudaMemset(ctx->status, 0, small)) != cudaSuccess) {

@@ -25,6 +25,7 @@ struct AttnParams {
     float *part_stat;      // [B, Hkv, n_split, M, 4]: m (log2 units), l, l_vis, unused
     uint32_t *status;      // device status word
     int32_t B, gamma, Hq, Hkv, D, Lmax, G, M, n_split;
+    int32_t pdl;           // launch programmatically dependent on the previous kernel
     float scale_log2;      // log2(e) / sqrt(D)
 };
 

@@ -196,31 +196,65 @@ attn_simt_kernel(const AttnParams p, const SeqInfo seq)
 
 // Merge of the KV splits: one CTA per (sequence, KV head, row), one thread per
 // output channel.  Splits are merged in index order, so the result does not
-// depend on scheduling.
-__global__ void attn_combine_kernel(const AttnParams p)
+// depend on scheduling.  The kernel may be launched programmatically dependent
+// on the attention kernel: it lets the next launch be scheduled, then waits
+// for the partials.
+constexpr int kCombineBatch = 32;    // splits whose partials one thread keeps in flight
+
+__global__ void __launch_bounds__(128) attn_combine_kernel(const AttnParams p)
 {
+    __shared__ float4 stat_s[kCombineBatch];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int r = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
     const int d = threadIdx.x;
     const int M = p.M, D = p.D, ns = p.n_split;
     const size_t unit0 = ((size_t)b * p.Hkv + kvh) * ns;
     const float *ps = p.part_stat + unit0 * (size_t)M * 4 + r * 4;
+    const float *po = p.part_o + (unit0 * (size_t)M + r) * D + (d < D ? d : 0);
+    const size_t o_stride = (size_t)M * D;
 
-    float m_star = -INFINITY;
-    for (int s = 0; s < ns; ++s) m_star = fmaxf(m_star, ps[(size_t)s * M * 4]);
-    float l = 0.f, lv = 0.f, o = 0.f;
-    for (int s = 0; s < ns; ++s) {
-        const float4 st = *reinterpret_cast<const float4 *>(ps + (size_t)s * M * 4);
-        if (st.y > 0.f) {
-            const float w = exp2f(st.x - m_star);
-            l = fmaf(w, st.y, l);
-            lv = fmaf(w, st.z, lv);
-            o = fmaf(w, p.part_o[((unit0 + s) * (size_t)M + r) * D + d], o);
+    // Batches of 32 splits: the statistics and the partial outputs of a batch are
+    // all requested before any is used (one round trip to L2 per batch).  The
+    // running reference exponent m_run moves up between batches like an online
+    // softmax; within a batch the splits are merged in index order.
+    float m_run = -INFINITY, l = 0.f, lv = 0.f, o = 0.f;
+    for (int s0 = 0; s0 < ns; s0 += kCombineBatch) {
+        const int n = min(kCombineBatch, ns - s0);
+        float v[kCombineBatch];
+#pragma unroll
+        for (int u = 0; u < kCombineBatch; ++u)
+            v[u] = u < n ? __ldcg(po + (size_t)(s0 + u) * o_stride) : 0.f;
+        __syncthreads();
+        if (threadIdx.x < n)
+            stat_s[threadIdx.x] =
+                __ldcg(reinterpret_cast<const float4 *>(ps + (size_t)(s0 + threadIdx.x) * M * 4));
+        __syncthreads();
+        float m_b = m_run;
+        for (int u = 0; u < n; ++u)
+            if (stat_s[u].y > 0.f) m_b = fmaxf(m_b, stat_s[u].x);
+        if (m_b > m_run) {
+            const float c = exp2f(m_run - m_b);     // 0 on the first batch
+            l *= c; lv *= c; o *= c;
+            m_run = m_b;
+        }
+#pragma unroll
+        for (int u = 0; u < kCombineBatch; ++u) {
+            if (u < n) {
+                const float4 st = stat_s[u];
+                if (st.y > 0.f) {
+                    const float w = exp2f(st.x - m_run);
+                    l = fmaf(w, st.y, l);
+                    lv = fmaf(w, st.z, lv);
+                    o = fmaf(w, v[u], o);
+                }
+            }
         }
     }
     const float inv = 1.f / l;
     const int g = r / p.G, hg = r - g * p.G;
     const size_t row = ((size_t)b * p.gamma + g) * p.Hq + kvh * p.G + hg;
-    reinterpret_cast<__nv_bfloat16 *>(p.out)[row * D + d] = __float2bfloat16_rn(o * inv);
+    if (d < D) reinterpret_cast<__nv_bfloat16 *>(p.out)[row * D + d] = __float2bfloat16_rn(o * inv);
     if (d == 0) p.mass[row] = lv * inv;
 }
 
@@ -251,10 +285,18 @@ cudaError_t launch_attn_simt(const AttnParams &p, const SeqInfo &seq, cudaStream
 
 cudaError_t launch_attn_combine(const AttnParams &p, cudaStream_t stream, int *launches)
 {
-    dim3 grid(p.M, p.Hkv, p.B);
-    attn_combine_kernel<<<grid, p.D, 0, stream>>>(p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.M, p.Hkv, p.B);
+    cfg.blockDim = dim3(128, 1, 1);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 0;   // an early-launched combine grid piles up on the few idle SMs: plain launch
+    cudaError_t err = cudaLaunchKernelEx(&cfg, attn_combine_kernel, p);
     ++*launches;
-    return cudaGetLastError();
+    return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 }  // namespace lvspec

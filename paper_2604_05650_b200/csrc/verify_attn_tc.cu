@@ -283,6 +283,8 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         }
         fence_proxy_async_smem();
     }
+    // nobody polls a barrier while the grid before this one is still running
+    grid_dependency_wait();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -662,10 +664,19 @@ cudaError_t launch_attn_tc(const AttnParams &p, const SeqInfo &seq, cudaStream_t
     cudaError_t err = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)smem);
     if (err != cudaSuccess) return err;
-    dim3 grid(p.n_split, p.Hkv, p.B);
-    attn_tc_kernel<<<grid, kThreads, smem, stream>>>(P, seq, mk, mv, mq);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.n_split, p.Hkv, p.B);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = p.pdl ? 1 : 0;
+    err = cudaLaunchKernelEx(&cfg, attn_tc_kernel, P, seq, mk, mv, mq);
     ++*launches;
-    return cudaGetLastError();
+    return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 }  // namespace lvspec
