@@ -112,7 +112,7 @@ __device__ __forceinline__ bool group_any(int id, bool pred)
 
 // exp2 of eight scaled scores of one position, packed to bf16; returns their maximum
 __device__ __forceinline__ float exp_chunk(const uint32_t (&r)[8], const float *m8, float scale,
-                                           bool tail, int col0, int G, int gmin, uint4 *dst)
+                                           bool tail, int col0, int G, int gmin, uint4 &dst)
 {
     const float4 ma = *reinterpret_cast<const float4 *>(m8);
     const float4 mb = *reinterpret_cast<const float4 *>(m8 + 4);
@@ -131,7 +131,7 @@ __device__ __forceinline__ float exp_chunk(const uint32_t (&r)[8], const float *
     pk.y = pack_bf16x2(ex2(x[2]), ex2(x[3]));
     pk.z = pack_bf16x2(ex2(x[4]), ex2(x[5]));
     pk.w = pack_bf16x2(ex2(x[6]), ex2(x[7]));
-    *dst = pk;
+    dst = pk;
     return mx;
 }
 
@@ -295,16 +295,33 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             int nk = first_k, nv = first_v;   // loads issued so far
+            // K and V slots free up at different times: poll both, never block on one
+            uint64_t idle_since = 0;
+            uint32_t spin = 0;
             while (nk < T || nv < T) {
-                if (nk < T) {
-                    if (!mbar_wait(k_empty(nk % cfg.ks), ((nk / cfg.ks) - 1) & 1, abort_flag)) break;
+                bool progress = false;
+                if (nk < T && mbar_test_wait(k_empty(nk % cfg.ks), ((nk / cfg.ks) - 1) & 1)) {
                     load_k(nk);
                     ++nk;
+                    progress = true;
                 }
-                if (nv < T) {
-                    if (!mbar_wait(v_empty(nv % cfg.vs), ((nv / cfg.vs) - 1) & 1, abort_flag)) break;
+                if (nv < T && mbar_test_wait(v_empty(nv % cfg.vs), ((nv / cfg.vs) - 1) & 1)) {
                     load_v(nv);
                     ++nv;
+                    progress = true;
+                }
+                if (progress) {
+                    idle_since = 0;
+                } else {
+                    if (*abort_flag) break;
+                    if ((++spin & 255u) == 0) {
+                        const uint64_t now = global_timer_ns();
+                        if (idle_since == 0) idle_since = now;
+                        else if (now - idle_since > 2000000000ull) {
+                            *abort_flag = 1;
+                            break;
+                        }
+                    }
                 }
             }
             if (*abort_flag) {
@@ -439,35 +456,26 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             }
             const bool tail = pos0 + kTilePos > L - gamma;
             const int gmin = pos - L + gamma;           // queries g < gmin do not see `pos`
-            if (tail && grp == 0) {
-                // slots at or beyond kv_len hold whatever the cache holds: zero their V
-                // rows so that 0 * junk cannot poison the accumulators
-                mbar_wait(v_full(i % cfg.vs), (i / cfg.vs) & 1, abort_flag);
-                if (pos >= L) {
-                    uint8_t *vrow = gbase + sm.v + (i % cfg.vs) * kSlotBytes + row * 128;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        *reinterpret_cast<uint4 *>(vrow + c * 16) = make_uint4(0, 0, 0, 0);
-                        *reinterpret_cast<uint4 *>(vrow + kBoxBytes + c * 16) = make_uint4(0, 0, 0, 0);
-                    }
-                }
-            }
-            if (i >= cfg.pb) mbar_wait(p_free(pb), ((i / cfg.pb) - 1) & 1, abort_flag);
             uint8_t *prow = gbase + sm.p + pb * (NP * 256) + row * 16;
+            uint4 pk[8];   // this position's probabilities, 8 columns per entry
 
             for (int attempt = 0; attempt < 3; ++attempt) {
                 float gmax = -INFINITY;
-                for (int c8 = c_lo; c8 < c_hi; c8 += 2) {
-                    uint32_t r0[8], r1[8];
-                    const bool two = c8 + 1 < c_hi;
-                    tmem_ld_x8(s_addr + c8 * 8, r0);
-                    if (two) tmem_ld_x8(s_addr + c8 * 8 + 8, r1);
-                    tmem_wait_ld();
-                    gmax = fmaxf(gmax, exp_chunk(r0, m_s + c8 * 8, scale, tail, c8 * 8, G, gmin,
-                                                 reinterpret_cast<uint4 *>(prow + c8 * 2048)));
-                    if (two)
-                        gmax = fmaxf(gmax, exp_chunk(r1, m_s + c8 * 8 + 8, scale, tail, c8 * 8 + 8, G, gmin,
-                                                     reinterpret_cast<uint4 *>(prow + (c8 + 1) * 2048)));
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int cb = c_lo + 4 * h;
+                    if (cb < c_hi) {
+                        uint32_t r[4][8];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (cb + u < c_hi) tmem_ld_x8(s_addr + (cb + u) * 8, r[u]);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (cb + u < c_hi)
+                                gmax = fmaxf(gmax, exp_chunk(r[u], m_s + (cb + u) * 8, scale, tail,
+                                                             (cb + u) * 8, G, gmin, pk[4 * h + u]));
+                    }
                 }
                 if (!group_any(bar_id, gmax > kGuard)) break;
 
@@ -523,15 +531,31 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 }
                 group_sync(bar_id);
             }
-            // S^T has been read and P^T (with any zeroed V rows) is in shared memory:
-            // one arrival per warp tells the MMA warp
+            // S^T has been read: the next K.Q^T may overwrite this buffer
             tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(s_free(sb));
+            if (tail && grp == 0) {
+                // slots at or beyond kv_len hold whatever the cache holds: zero their V
+                // rows so that 0 * junk cannot poison the accumulators
+                mbar_wait(v_full(i % cfg.vs), (i / cfg.vs) & 1, abort_flag);
+                if (pos >= L) {
+                    uint8_t *vrow = gbase + sm.v + (i % cfg.vs) * kSlotBytes + row * 128;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        *reinterpret_cast<uint4 *>(vrow + c * 16) = make_uint4(0, 0, 0, 0);
+                        *reinterpret_cast<uint4 *>(vrow + kBoxBytes + c * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                }
+            }
+            // P^T goes to shared memory once the P.V product that read this buffer is done
+            if (i >= cfg.pb) mbar_wait(p_free(pb), ((i / cfg.pb) - 1) & 1, abort_flag);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (c_lo + j < c_hi) *reinterpret_cast<uint4 *>(prow + (c_lo + j) * 2048) = pk[j];
             fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(s_free(sb));
-                mbar_arrive(p_full(pb));
-            }
+            if (lane == 0) mbar_arrive(p_full(pb));
         }
 
         // ---------------------------------------------------------------- epilogue
@@ -632,9 +656,10 @@ TcConfig pick_config(int M)
 {
     TcConfig c;
     c.n_pad = (M + 15) & ~15;
-    // deepest K/V rings that fit, two P buffers before a third V slot is given up
-    const int tries[4][3] = {{2, 3, 2}, {2, 3, 1}, {2, 2, 2}, {2, 2, 1}};
-    for (int t = 0; t < 4; ++t) {
+    // deepest K/V rings that fit: bytes in flight matter more than a second P buffer,
+    // since the probabilities wait in registers for the buffer anyway
+    const int tries[6][3] = {{3, 3, 2}, {3, 3, 1}, {2, 3, 2}, {2, 3, 1}, {2, 2, 2}, {2, 2, 1}};
+    for (int t = 0; t < 6; ++t) {
         c.ks = tries[t][0]; c.vs = tries[t][1]; c.pb = tries[t][2];
         if (smem_map(c).total <= kMaxSmem) break;
     }
