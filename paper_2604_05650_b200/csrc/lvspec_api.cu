@@ -192,6 +192,8 @@ lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, con
     }
     ctx->launches += launches;
     if (e != cudaSuccess) return cuda_fail(ctx, "attention kernel launch", e);
+    // with a single split the tensor-core kernel writes the results itself
+    if (kernel == LVSPEC_KERNEL_TCGEN05 && p.n_split == 1) return LVSPEC_OK;
     launches = 0;
     e = launch_attn_combine(p, ctx->stream, &launches);
     ctx->launches += launches;

@@ -150,8 +150,9 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
 
     // tiles [t_begin, t_begin + T) of this split: equal shares, sizes differ by at most one
     const int n_tiles = (L + kTilePos - 1) / kTilePos;
-    const int t_begin = (int)(((long long)split * n_tiles) / p.n_split);
-    const int T = (int)(((long long)(split + 1) * n_tiles) / p.n_split) - t_begin;
+    const int t_base = n_tiles / p.n_split, t_rem = n_tiles - t_base * p.n_split;
+    const int t_begin = split * t_base + min(split, t_rem);
+    const int T = t_base + (split < t_rem ? 1 : 0);
 
     const size_t unit = ((size_t)b * p.Hkv + kvh) * p.n_split + split;
     float *part_o = p.part_o + unit * (size_t)M * 128;
@@ -211,12 +212,13 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     int first_k = 0, first_v = 0;   // loads issued before the CTA-wide barrier
     if (warp == 0) {
         if (lane == 0) {
-            for (int s = 0; s < cfg.ks; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); }
-            for (int s = 0; s < cfg.vs; ++s) { mbar_init(v_full(s), 1); mbar_init(v_empty(s), 1); }
-            for (int s = 0; s < 2; ++s) { mbar_init(s_full(s), 1); mbar_init(s_free(s), 8); }
-            for (int s = 0; s < cfg.pb; ++s) { mbar_init(p_full(s), 8); mbar_init(p_free(s), 1); }
-            mbar_init(drain_bar, 1);
-            mbar_init(done_bar, 9);
+            // the TMA unit fetches the descriptors while the barriers are set up
+            prefetch_tensormap(&tmap_k);
+            prefetch_tensormap(&tmap_v);
+            prefetch_tensormap(&tmap_q);
+            // first the barriers the loads complete on, so that the loads can go out
+            for (int s = 0; s < cfg.ks; ++s) mbar_init(k_full(s), 1);
+            for (int s = 0; s < cfg.vs; ++s) mbar_init(v_full(s), 1);
             mbar_init(q_full, 1);
             *abort_flag = 0;
             mbar_fence_init();
@@ -232,6 +234,13 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 if (i < first_k) load_k(i);
                 load_v(i);
             }
+            for (int s = 0; s < cfg.ks; ++s) mbar_init(k_empty(s), 1);
+            for (int s = 0; s < cfg.vs; ++s) mbar_init(v_empty(s), 1);
+            for (int s = 0; s < 2; ++s) { mbar_init(s_full(s), 1); mbar_init(s_free(s), 8); }
+            for (int s = 0; s < cfg.pb; ++s) { mbar_init(p_full(s), 8); mbar_init(p_free(s), 1); }
+            mbar_init(drain_bar, 1);
+            mbar_init(done_bar, 9);
+            mbar_fence_init();
             grid_launch_dependents();
         }
         __syncwarp();
@@ -395,11 +404,12 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 if (uniform >= 0) {
                     const uint64_t d2 = a2d0 + (uint64_t)(uniform * (kA2Bytes >> 4));
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const uint32_t acc = j > 0 ? 1u : first_acc;
-                        mma_f16_ss(tm_o, vd + (uint64_t)(j * 128), pd + (uint64_t)(j * 16), idesc_pv, acc);
-                        mma_f16_ss(tm_l, d2, pd + (uint64_t)(j * 16), idesc_sum, acc);
-                    }
+                    for (int j = 0; j < 8; ++j)
+                        mma_f16_ss(tm_l, d2, pd + (uint64_t)(j * 16), idesc_sum, j > 0 ? 1u : first_acc);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        mma_f16_ss(tm_o, vd + (uint64_t)(j * 128), pd + (uint64_t)(j * 16), idesc_pv,
+                                   j > 0 ? 1u : first_acc);
                 } else {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
@@ -561,25 +571,74 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         // ---------------------------------------------------------------- epilogue
         mbar_wait(p_free((T - 1) % cfg.pb), ((T - 1) / cfg.pb) & 1, abort_flag);
         tc_fence_after();
-        for (int c8 = c_lo; c8 < c_hi; ++c8) {
-            uint32_t r[8];
-            tmem_ld_x8(tm_o + lane_addr + c8 * 8, r);
-            tmem_wait_ld();
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const int n = c8 * 8 + k;
-                if (n < M) part_o[(size_t)n * 128 + row] = __uint_as_float(r[k]);
-            }
+        if (p.n_split == 1) {
+            // a single split: nothing to merge, normalise and write the results here
             if (wq == 0) {
-                tmem_ld_x8(tm_l + c8 * 8, r);     // lane 0: l, lane 1: l_vis
+                for (int c8 = c_lo; c8 < c_hi; ++c8) {
+                    uint32_t r[8];
+                    tmem_ld_x8(tm_l + c8 * 8, r);     // lane 0: l, lane 1: l_vis
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const int n = c8 * 8 + k;
+                        const float lv = __shfl_sync(0xffffffffu, __uint_as_float(r[k]), 1);
+                        if (lane == 0 && n < M) {
+                            const float inv = 1.f / __uint_as_float(r[k]);
+                            dl_s[n] = inv;
+                            const int g = n / G, hg = n - g * G;
+                            p.mass[((size_t)b * gamma + g) * p.Hq + kvh * G + hg] = lv * inv;
+                        }
+                    }
+                }
+            }
+            group_sync(bar_id);
+            __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(p.out);
+            for (int c8 = c_lo; c8 < c_hi; ++c8) {
+                uint32_t r[8];
+                tmem_ld_x8(tm_o + lane_addr + c8 * 8, r);
                 tmem_wait_ld();
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
                     const int n = c8 * 8 + k;
-                    const float lv = __shfl_sync(0xffffffffu, __uint_as_float(r[k]), 1);
-                    if (lane == 0 && n < M)
-                        *reinterpret_cast<float4 *>(part_stat + n * 4) =
-                            make_float4(m_s[n], __uint_as_float(r[k]), lv, 0.f);
+                    if (n < M) {
+                        const int g = n / G, hg = n - g * G;
+                        out[(((size_t)b * gamma + g) * p.Hq + kvh * G + hg) * 128 + row] =
+                            __float2bfloat16_rn(__uint_as_float(r[k]) * dl_s[n]);
+                    }
+                }
+            }
+        } else {
+            // partial O^T: up to four chunks of 8 columns in flight per wait
+            for (int cb = c_lo; cb < c_hi; cb += 4) {
+                uint32_t r[4][8];
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (cb + u < c_hi) tmem_ld_x8(tm_o + lane_addr + (cb + u) * 8, r[u]);
+                tmem_wait_ld();
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (cb + u < c_hi) {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            const int n = (cb + u) * 8 + k;
+                            if (n < M) part_o[(size_t)n * 128 + row] = __uint_as_float(r[u][k]);
+                        }
+                    }
+                }
+            }
+            if (wq == 0) {
+                for (int c8 = c_lo; c8 < c_hi; ++c8) {
+                    uint32_t r[8];
+                    tmem_ld_x8(tm_l + c8 * 8, r);     // lane 0: l, lane 1: l_vis
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const int n = c8 * 8 + k;
+                        const float lv = __shfl_sync(0xffffffffu, __uint_as_float(r[k]), 1);
+                        if (lane == 0 && n < M)
+                            *reinterpret_cast<float4 *>(part_stat + n * 4) =
+                                make_float4(m_s[n], __uint_as_float(r[k]), lv, 0.f);
+                    }
                 }
             }
         }

@@ -205,3 +205,11 @@ def test_invalid_arguments_launch_nothing(ctx):
     with pytest.raises(binding.LvspecError):
         ctx.verify_attention(s, q.data_ptr() + 2, kv, kv, (256,), ((0, 10),), out, mass)
     assert ctx.launch_count() == before
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_sweep_point_single_split(ctx, oracle_mod, kernel):
+    """Batch 16 x 8 KV heads fills the device with one split per head: the
+    tensor-core kernel then normalises and writes the results itself."""
+    cfg = W.sweep_config(gamma=4, kv_len=4096, batch=16, point=9)
+    _check(ctx, oracle_mod, W.attention_inputs(cfg), kernel=kernel)
