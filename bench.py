@@ -36,7 +36,7 @@ UNIT = "tokens/s"
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="BASELINE config id (1, 2 or 3)")
@@ -44,6 +44,9 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch layer by layer, no CUDA graph")
+    ap.add_argument("--sweep", action="store_true",
+                    help="run the head-shape sweep (BASELINE config 4): gamma x KV length x batch, one layer "
+                         "per point; the JSON line then carries the per-point table under \"sweep\"")
     ap.add_argument("--layers", type=int, default=0,
                     help="override the config's layer count (a smaller case of the same kernel for "
                          "profiler captures; the line then says so and is not a bench value)")
@@ -54,32 +57,70 @@ def parse():
 # clocks
 # --------------------------------------------------------------------------- #
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed
-    region runs (reads settings only)."""
+    """Samples the SM clock and the throttle reasons while the timed region runs.
+    Reads only: NVML queries every few milliseconds (nvidia-smi as a fallback,
+    which is slower per sample)."""
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, index: int):
         self.index = index
-        self.samples = []
+        self.samples = []          # (sm_mhz, max_mhz, [bool per NAMES])
         self._stop = threading.Event()
         self._thread = None
+        self._nvml = None
+        self._handle = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._handle = self._pick_handle(pynvml, index)
+            self._nvml = pynvml
+            self._max = float(pynvml.nvmlDeviceGetMaxClockInfo(self._handle, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nvml = None
+
+    @staticmethod
+    def _pick_handle(pynvml, index):
+        # CUDA_VISIBLE_DEVICES may renumber the devices: go by UUID when it names one
+        vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+        ids = [x.strip() for x in vis.split(",") if x.strip()]
+        if index < len(ids):
+            tok = ids[index]
+            if tok.startswith("GPU-"):
+                return pynvml.nvmlDeviceGetHandleByUUID(tok)
+            if tok.isdigit():
+                return pynvml.nvmlDeviceGetHandleByIndex(int(tok))
+        return pynvml.nvmlDeviceGetHandleByIndex(index)
 
     def _once(self):
         try:
+            if self._nvml is not None:
+                n = self._nvml
+                sm = float(n.nvmlDeviceGetClockInfo(self._handle, n.NVML_CLOCK_SM))
+                r = int(n.nvmlDeviceGetCurrentClocksEventReasons(self._handle)) \
+                    if hasattr(n, "nvmlDeviceGetCurrentClocksEventReasons") \
+                    else int(n.nvmlDeviceGetCurrentClocksThrottleReasons(self._handle))
+                flags = [bool(r & n.nvmlClocksThrottleReasonHwSlowdown),
+                         bool(r & n.nvmlClocksThrottleReasonHwThermalSlowdown),
+                         bool(r & n.nvmlClocksThrottleReasonSwThermalSlowdown),
+                         bool(r & n.nvmlClocksThrottleReasonSwPowerCap)]
+                self.samples.append((sm, self._max, flags))
+                return
             out = subprocess.run(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
                                   "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
             parts = [x.strip() for x in out.strip().split(",")]
             if len(parts) >= 6:
-                self.samples.append(parts)
+                self.samples.append((float(parts[0]), float(parts[1]),
+                                     [x.lower() == "active" for x in parts[2:6]]))
         except Exception:
             pass
 
     def _run(self):
         while not self._stop.is_set():
             self._once()
-            self._stop.wait(0.1)
+            self._stop.wait(0.002 if self._nvml is not None else 0.1)
 
     def start(self):
         self._thread = threading.Thread(target=self._run, daemon=True)
@@ -93,12 +134,12 @@ class ClockSampler:
             self._once()
 
     def summary(self):
-        sm = [float(s[0]) for s in self.samples if s[0].replace(".", "").isdigit()]
-        mx = [float(s[1]) for s in self.samples if s[1].replace(".", "").isdigit()]
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [n for i, n in enumerate(names) if any(s[2 + i].lower() == "active" for s in self.samples)]
+        sm = [s[0] for s in self.samples]
+        mx = [s[1] for s in self.samples]
+        reasons = [n for i, n in enumerate(self.NAMES) if any(s[2][i] for s in self.samples)]
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(self.samples)}
+                "sm_mhz_min": min(sm) if sm else None, "reasons": reasons, "samples": len(self.samples),
+                "source": "nvml" if self._nvml is not None else "nvidia-smi"}
 
 
 # --------------------------------------------------------------------------- #
@@ -400,8 +441,114 @@ def run_e2e(args, cfg, ctx, stream, qs, ks, vs_, logits, draft, torch, dev, worl
             "note": "K/V caches of every layer cross PCIe each step"}
 
 
+def run_sweep(args):
+    """BASELINE config 4: the 40/8x128 head shape, one layer, gamma x KV length x
+    batch.  Per point: time of one attention call and of the acceptance pass,
+    achieved HBM GB/s of the attention call against the measured peak, verified
+    tokens/s of the single-layer step.  Each point rotates over enough distinct
+    K/V buffers (>= 256 MB in total, at least 2) that no call finds its cache in L2."""
+    import torch
+    from paper_2604_05650_b200 import binding, build as _build, workloads as W
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    _build.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    ctx = binding.Context(0)
+    stream = torch.cuda.Stream(device=dev)
+    ctx.set_stream(stream.cuda_stream)
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak = float(json.load(open(peaks_path))["hbm_gbs"]) if os.path.exists(peaks_path) else 6650.0
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(4)
+    points, tok_total, ms_total = [], 0.0, 0.0
+    clocks = ClockSampler(0)
+    clocks.start()
+    idx = 0
+    for batch in W.SWEEP_BATCHES:
+        for kv in W.SWEEP_KV_LENS:
+            kv_bytes = 2 * batch * 8 * kv * 128 * 2
+            copies = max(2, -(-(256 << 20) // kv_bytes))
+            ks = [torch.randn((batch, 8, kv, 128), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+                  for _ in range(copies)]
+            vs_ = [torch.randn((batch, 8, kv, 128), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+                   for _ in range(copies)]
+            for gamma in W.SWEEP_GAMMAS:
+                cfg = W.sweep_config(gamma=gamma, kv_len=kv, batch=batch, point=idx)
+                idx += 1
+                logits_h, draft_h = W.accept_inputs(cfg)
+                logits, draft = torch.from_numpy(logits_h).to(dev), torch.from_numpy(draft_h).to(dev)
+                q = torch.randn((batch, gamma, 40, 128), generator=gen, device=dev).to(torch.bfloat16)
+                out = torch.empty_like(q)
+                mass = torch.empty((batch, gamma, 40), dtype=torch.float32, device=dev)
+                alen = torch.zeros((batch,), dtype=torch.int32, device=dev)
+                shape = binding.attn_shape(batch, gamma, 40, 8, 128, kv, 0, args.kernel)
+                kv_len = np.full((batch,), kv, dtype=np.int32)
+                span = np.tile(np.asarray([cfg.span], dtype=np.int32), (batch, 1))
+
+                def rotation():
+                    for c in range(copies):
+                        ctx.verify_attention(shape, q, ks[c], vs_[c], kv_len, span, out, mass)
+
+                def accept():
+                    ctx.loose_accept(batch, gamma, cfg.vocab, 40, logits, draft, mass, alen,
+                                     cfg.shift_window, lam=cfg.lam)
+
+                with torch.cuda.stream(stream):
+                    rotation()
+                    accept()
+                stream.synchronize()
+                g_attn, g_acc = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g_attn, stream=stream):
+                    rotation()
+                with torch.cuda.graph(g_acc, stream=stream):
+                    accept()
+                reps = max(3, min(50, int(2000 // copies)))
+                e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+                with torch.cuda.stream(stream):
+                    for _ in range(3):
+                        g_attn.replay()
+                        g_acc.replay()
+                    e0.record(stream)
+                    for _ in range(reps):
+                        g_attn.replay()
+                    e1.record(stream)
+                    for _ in range(reps):
+                        g_acc.replay()
+                    e2.record(stream)
+                stream.synchronize()
+                us_attn = e0.elapsed_time(e1) * 1e3 / (reps * copies)
+                us_acc = e1.elapsed_time(e2) * 1e3 / reps
+                nbytes = kv_bytes + 2 * q.numel() * 2 + mass.numel() * 4
+                gbs = nbytes / (us_attn * 1e-6) / 1e9
+                tps = batch * gamma / ((us_attn + us_acc) * 1e-6)
+                points.append({"batch": batch, "kv_len": kv, "gamma": gamma, "us_attention": round(us_attn, 2),
+                               "us_accept": round(us_acc, 2), "hbm_gbs": round(gbs, 1),
+                               "frac_of_measured_peak": round(gbs / peak, 4), "tokens_per_s": round(tps, 1),
+                               "splits": ctx.attention_splits(shape, kv), "kv_buffers": copies})
+                tok_total += batch * gamma
+                ms_total += (us_attn + us_acc) * 1e-3
+                del g_attn, g_acc
+            del ks, vs_
+            torch.cuda.empty_cache()
+    clocks.stop()
+    status = ctx.device_status()
+    ctx.close()
+    line = {"metric": METRIC, "value": tok_total / (ms_total * 1e-3), "unit": UNIT, "n_gpus": 1,
+            "steps": len(points), "warmup": 3, "ms_per_step": ms_total / len(points), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "BASELINE config 4: sweep on the 40/8x128 head shape, one layer per point, "
+                                   "gamma {4,8,16} x KV {4K,16K,64K,128K} x batch {1,4,16}, 75% visual",
+                       "l2": "each point rotates over >= 256 MB of distinct K/V buffers"},
+            "device_status": status, "clocks": clocks.summary(), "peak_hbm_gbs": peak, "sweep": points}
+    print(json.dumps(line))
+
+
 def main():
     args = parse()
+    if args.sweep:
+        run_sweep(args)
+        return
     from paper_2604_05650_b200 import workloads as W
     cfg = W.CONFIGS[args.config]
     if args.layers > 0:
