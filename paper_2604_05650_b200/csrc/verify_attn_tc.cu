@@ -18,13 +18,13 @@
 // reduction in this layout) and the accumulators rescaled.  fp32 and bf16
 // share the exponent range, so nothing is lost in between.
 //
-// Warp roles (352 threads): warp 0 = TMA producer, warp 1 = issuer of the
-// K.Q^T MMAs and TMEM owner, warp 10 = issuer of the P.V and sum MMAs (one
+// Warp roles (480 threads): warp 0 = TMA producer, warp 1 = issuer of the
+// K.Q^T MMAs and TMEM owner, warp 14 = issuer of the P.V and sum MMAs (one
 // thread each; two issuers because a single thread's issue rate, not the tensor
-// pipe, bounded the loop), warps 2-5 and 6-9 = two softmax groups.  Both groups work on
-// every tile, each on its own half of the N columns (TMEM lane quarter = warp
-// % 4), so the two halves never interact: each has its own m, its own guard
-// and its own rescale.  K and V tiles sit in separate shared-memory rings,
+// pipe, bounded the loop), warps 2-13 = three softmax groups of four warps.
+// All groups work on every tile, each on its own share of the N columns (TMEM
+// lane quarter = warp % 4), so the shares never interact: each has its own m,
+// its own guard and its own rescale.  K and V tiles sit in separate shared-memory rings,
 // each slot two 128-position x 64-channel boxes with the 128-byte swizzle; Q
 // arrives by TMA in the same layout.  Every mbarrier wait is bounded; a wait
 // that gives up raises LVSPEC_DEV_WAIT_EXPIRED.
@@ -40,9 +40,13 @@ namespace {
 using namespace ptx;
 
 constexpr int kTilePos = 128;
-constexpr int kThreads = 352;
-constexpr int kPvWarp = 10;                 // issues the P.V and sum MMAs
+constexpr int kSoftmaxGroups = 3;           // groups of 4 warps, each on its own share of the columns
 constexpr int kSoftmaxWarp0 = 2;            // first softmax warp
+constexpr int kSoftmaxWarps = 4 * kSoftmaxGroups;
+constexpr int kSoftmaxThreads = 32 * kSoftmaxWarps;
+constexpr int kPvWarp = kSoftmaxWarp0 + kSoftmaxWarps;   // issues the P.V and sum MMAs
+constexpr int kThreads = 32 * (kPvWarp + 1);
+constexpr int kMaxChunks = (LVSPEC_MAX_ROWS / 8 + kSoftmaxGroups - 1) / kSoftmaxGroups;   // per group
 constexpr uint32_t kBoxBytes = 16384;       // 128 positions x 64 channels bf16
 constexpr uint32_t kSlotBytes = 2 * kBoxBytes;
 constexpr uint32_t kA2Bytes = 2048;         // one 64 x 16 constant tile
@@ -91,7 +95,7 @@ __device__ __forceinline__ bool wait_unconditional(uint32_t bar, uint32_t parity
     return true;
 }
 
-// named barrier over the 128 threads of one softmax group (ids 1 and 2)
+// named barrier over the 128 threads of one softmax group (ids 1, 2, ...)
 __device__ __forceinline__ void group_sync(int id)
 {
     asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory");
@@ -236,10 +240,10 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             }
             for (int s = 0; s < cfg.ks; ++s) mbar_init(k_empty(s), 1);
             for (int s = 0; s < cfg.vs; ++s) mbar_init(v_empty(s), 1);
-            for (int s = 0; s < 2; ++s) { mbar_init(s_full(s), 1); mbar_init(s_free(s), 8); }
-            for (int s = 0; s < cfg.pb; ++s) { mbar_init(p_full(s), 8); mbar_init(p_free(s), 1); }
+            for (int s = 0; s < 2; ++s) { mbar_init(s_full(s), 1); mbar_init(s_free(s), kSoftmaxWarps); }
+            for (int s = 0; s < cfg.pb; ++s) { mbar_init(p_full(s), kSoftmaxWarps); mbar_init(p_free(s), 1); }
             mbar_init(drain_bar, 1);
-            mbar_init(done_bar, 9);
+            mbar_init(done_bar, kSoftmaxWarps + 1);
             mbar_fence_init();
             grid_launch_dependents();
         }
@@ -248,23 +252,23 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         tmem_alloc(base + sm.misc, (uint32_t)cfg.tmem_cols);
         tmem_relinquish();
     } else if (warp < kPvWarp) {
-        const int idx = tid - 64;   // 0..255
+        const int idx = tid - 64;   // 0..kSoftmaxThreads-1
         // rows M..NP-1 of Q are padding: zero them (the TMA boxes cover rows < M only)
-        for (int i = idx; i < (NP - M) * 16; i += 256) {
+        for (int i = idx; i < (NP - M) * 16; i += kSoftmaxThreads) {
             const int r = M + (i >> 4), c = i & 15, h = c >> 3, cc = c & 7;
             *reinterpret_cast<uint4 *>(gbase + sm.q + h * (NP * 128) + r * 128 + cc * 16) =
                 make_uint4(0, 0, 0, 0);
         }
         // P buffers start as zeros (columns beyond the last chunk stay zero)
-        for (uint32_t i = idx * 16; i < (uint32_t)(cfg.pb * NP * 256); i += 256 * 16)
+        for (uint32_t i = idx * 16; i < (uint32_t)(cfg.pb * NP * 256); i += kSoftmaxThreads * 16)
             *reinterpret_cast<uint4 *>(gbase + sm.p + i) = make_uint4(0, 0, 0, 0);
-        for (int n = idx; n < NP; n += 256) m_s[n] = 0.f;
+        for (int n = idx; n < NP; n += kSoftmaxThreads) m_s[n] = 0.f;
         // constant 64 x 16 tiles (K-major, no swizzle: the 8 positions of chunk c
         // at c * 1024, row r at (r / 8) * 128 + (r % 8) * 16).  Row 0 = ones (sums
         // l), row 1 = 1 inside the visual span (sums l_vis), rows 2.. = 0.
         // tile 0: block inside the span, 1: outside, 2: the 16-block holding the
         // span start, 3: the 16-block holding the span end
-        for (uint32_t i = idx * 16; i < 4 * kA2Bytes; i += 256 * 16) {
+        for (uint32_t i = idx * 16; i < 4 * kA2Bytes; i += kSoftmaxThreads * 16) {
             const int tile = i / kA2Bytes, off = i % kA2Bytes;
             const int c = off / 1024, rr = (off % 1024) / 16;   // rr = row index 0..63
             uint4 val = make_uint4(0, 0, 0, 0);
@@ -439,13 +443,17 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         const int row = wq * 32 + lane;                 // TMEM lane = position inside the tile
         const int gtid = ((warp - kSoftmaxWarp0) & 3) * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
-        const int n_a = (n8 + 1) >> 1;
-        const int c_lo = grp ? n_a : 0, c_hi = grp ? n8 : n_a;   // chunks of 8 columns
+        // chunks of 8 columns [c_lo, c_hi) of this group: equal shares, at most kMaxChunks
+        const int c_base = n8 / kSoftmaxGroups, c_rem = n8 - c_base * kSoftmaxGroups;
+        const int c_lo = grp * c_base + min(grp, c_rem), c_hi = c_lo + c_base + (grp < c_rem ? 1 : 0);
         const float scale = p.scale_log2;
+        // ring positions advance by counting, not by dividing
+        int pb = 0, vsl = 0;                 // P buffer and V slot of tile i
+        uint32_t pb_round = 0, vs_round = 0; // how often each ring has wrapped
         for (int i = 0; i < T; ++i) {
             const int pos0 = (t_begin + i) * kTilePos;
             const int pos = pos0 + row;
-            const int sb = i & 1, pb = i % cfg.pb;
+            const int sb = i & 1;
             mbar_wait(s_full(sb), (i >> 1) & 1, abort_flag);
             tc_fence_after();
             const uint32_t s_addr = tm_s0 + sb * NP + lane_addr;
@@ -467,22 +475,22 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             const bool tail = pos0 + kTilePos > L - gamma;
             const int gmin = pos - L + gamma;           // queries g < gmin do not see `pos`
             uint8_t *prow = gbase + sm.p + pb * (NP * 256) + row * 16;
-            uint4 pk[8];   // this position's probabilities, 8 columns per entry
+            uint4 pk[kMaxChunks];   // this position's probabilities, 8 columns per entry
 
             for (int attempt = 0; attempt < 3; ++attempt) {
                 float gmax = -INFINITY;
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
+                for (int h = 0; h < (kMaxChunks + 3) / 4; ++h) {
                     const int cb = c_lo + 4 * h;
                     if (cb < c_hi) {
                         uint32_t r[4][8];
 #pragma unroll
                         for (int u = 0; u < 4; ++u)
-                            if (cb + u < c_hi) tmem_ld_x8(s_addr + (cb + u) * 8, r[u]);
+                            if (4 * h + u < kMaxChunks && cb + u < c_hi) tmem_ld_x8(s_addr + (cb + u) * 8, r[u]);
                         tmem_wait_ld();
 #pragma unroll
                         for (int u = 0; u < 4; ++u)
-                            if (cb + u < c_hi)
+                            if (4 * h + u < kMaxChunks && cb + u < c_hi)
                                 gmax = fmaxf(gmax, exp_chunk(r[u], m_s + (cb + u) * 8, scale, tail,
                                                              (cb + u) * 8, G, gmin, pk[4 * h + u]));
                     }
@@ -517,7 +525,12 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 if (i > 0) {
                     // O^T and the sums were accumulated under the old m: rescale this
                     // group's columns once PV(i-1) has finished
-                    mbar_wait(p_free((i - 1) % cfg.pb), ((i - 1) / cfg.pb) & 1, abort_flag);
+                    {
+                        // the P buffer of tile i - 1 and the round it was filled in
+                        const int pp = pb == 0 ? cfg.pb - 1 : pb - 1;
+                        const uint32_t pr = pb == 0 ? pb_round - 1 : pb_round;
+                        mbar_wait(p_free(pp), pr & 1, abort_flag);
+                    }
                     tc_fence_after();
                     for (int c8 = c_lo; c8 < c_hi; ++c8) {
                         uint32_t r[8];
@@ -541,16 +554,12 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 }
                 group_sync(bar_id);
             }
-            // S^T has been read: the next K.Q^T may overwrite this buffer
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(s_free(sb));
             if (tail && grp == 0) {
                 // slots at or beyond kv_len hold whatever the cache holds: zero their V
                 // rows so that 0 * junk cannot poison the accumulators
-                mbar_wait(v_full(i % cfg.vs), (i / cfg.vs) & 1, abort_flag);
+                mbar_wait(v_full(vsl), vs_round & 1, abort_flag);
                 if (pos >= L) {
-                    uint8_t *vrow = gbase + sm.v + (i % cfg.vs) * kSlotBytes + row * 128;
+                    uint8_t *vrow = gbase + sm.v + vsl * kSlotBytes + row * 128;
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         *reinterpret_cast<uint4 *>(vrow + c * 16) = make_uint4(0, 0, 0, 0);
@@ -559,17 +568,29 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 }
             }
             // P^T goes to shared memory once the P.V product that read this buffer is done
-            if (i >= cfg.pb) mbar_wait(p_free(pb), ((i / cfg.pb) - 1) & 1, abort_flag);
+            if (pb_round > 0) mbar_wait(p_free(pb), (pb_round - 1) & 1, abort_flag);
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
+            for (int j = 0; j < kMaxChunks; ++j)
                 if (c_lo + j < c_hi) *reinterpret_cast<uint4 *>(prow + (c_lo + j) * 2048) = pk[j];
+            // one arrival per warp: S^T has been read (the next K.Q^T but one may overwrite
+            // it) and P^T, with any zeroed V rows, is in shared memory
+            tc_fence_before();
             fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) mbar_arrive(p_full(pb));
+            if (lane == 0) {
+                mbar_arrive(s_free(sb));
+                mbar_arrive(p_full(pb));
+            }
+            if (++pb == cfg.pb) { pb = 0; ++pb_round; }
+            if (++vsl == cfg.vs) { vsl = 0; ++vs_round; }
         }
 
         // ---------------------------------------------------------------- epilogue
-        mbar_wait(p_free((T - 1) % cfg.pb), ((T - 1) / cfg.pb) & 1, abort_flag);
+        {
+            const int pp = pb == 0 ? cfg.pb - 1 : pb - 1;
+            const uint32_t pr = pb == 0 ? pb_round - 1 : pb_round;
+            mbar_wait(p_free(pp), pr & 1, abort_flag);
+        }
         tc_fence_after();
         if (p.n_split == 1) {
             // a single split: nothing to merge, normalise and write the results here
