@@ -194,68 +194,81 @@ attn_simt_kernel(const AttnParams p, const SeqInfo seq)
         *reinterpret_cast<float4 *>(ps + r * 4) = make_float4(m_s[r], l_s[r], lv_s[r], 0.f);
 }
 
-// Merge of the KV splits: one CTA per (sequence, KV head, row), one thread per
-// output channel.  Splits are merged in index order, so the result does not
+// Merge of the KV splits: one warp per (sequence, KV head, row), each lane four
+// output channels.  Splits are merged in index order, so the result does not
 // depend on scheduling.  The kernel may be launched programmatically dependent
 // on the attention kernel: it lets the next launch be scheduled, then waits
 // for the partials.
-constexpr int kCombineBatch = 32;    // splits whose partials one thread keeps in flight
+//
+// Batches of 32 splits: lane u fetches the statistics of split u while every
+// lane fetches its four channels of all 32 partial outputs, so a batch costs
+// one round trip to L2.  The running reference exponent moves up between
+// batches like an online softmax.
+constexpr int kCombineBatch = 32;
+constexpr int kCombineWarps = 4;
 
-__global__ void __launch_bounds__(128) attn_combine_kernel(const AttnParams p)
+__global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const AttnParams p)
 {
-    __shared__ float4 stat_s[kCombineBatch];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int r = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
-    const int d = threadIdx.x;
+    const int lane = threadIdx.x & 31;
+    const int r = blockIdx.x * kCombineWarps + (threadIdx.x >> 5), kvh = blockIdx.y, b = blockIdx.z;
     const int M = p.M, D = p.D, ns = p.n_split;
+    if (r >= M) return;
+    const bool active = lane * 4 < D;                   // D = 64 uses half the lanes
     const size_t unit0 = ((size_t)b * p.Hkv + kvh) * ns;
-    const float *ps = p.part_stat + unit0 * (size_t)M * 4 + r * 4;
-    const float *po = p.part_o + (unit0 * (size_t)M + r) * D + (d < D ? d : 0);
-    const size_t o_stride = (size_t)M * D;
+    const float4 *ps = reinterpret_cast<const float4 *>(p.part_stat) + unit0 * (size_t)M + r;
+    const float4 *po = reinterpret_cast<const float4 *>(p.part_o + (unit0 * (size_t)M + r) * D) +
+                       (active ? lane : 0);
+    const size_t o_stride = (size_t)M * D / 4;          // float4 units between splits
 
-    // Batches of 32 splits: the statistics and the partial outputs of a batch are
-    // all requested before any is used (one round trip to L2 per batch).  The
-    // running reference exponent m_run moves up between batches like an online
-    // softmax; within a batch the splits are merged in index order.
-    float m_run = -INFINITY, l = 0.f, lv = 0.f, o = 0.f;
+    float m_run = -INFINITY, l = 0.f, lv = 0.f;
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int s0 = 0; s0 < ns; s0 += kCombineBatch) {
         const int n = min(kCombineBatch, ns - s0);
-        float v[kCombineBatch];
+        float4 v[kCombineBatch];
 #pragma unroll
         for (int u = 0; u < kCombineBatch; ++u)
-            v[u] = u < n ? __ldcg(po + (size_t)(s0 + u) * o_stride) : 0.f;
-        __syncthreads();
-        if (threadIdx.x < n)
-            stat_s[threadIdx.x] =
-                __ldcg(reinterpret_cast<const float4 *>(ps + (size_t)(s0 + threadIdx.x) * M * 4));
-        __syncthreads();
-        float m_b = m_run;
-        for (int u = 0; u < n; ++u)
-            if (stat_s[u].y > 0.f) m_b = fmaxf(m_b, stat_s[u].x);
+            v[u] = u < n ? __ldcg(po + (size_t)(s0 + u) * o_stride) : make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 st = make_float4(-INFINITY, 0.f, 0.f, 0.f);
+        if (lane < n) st = __ldcg(ps + (size_t)(s0 + lane) * M);
+        float m_b = st.y > 0.f ? st.x : -INFINITY;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) m_b = fmaxf(m_b, __shfl_xor_sync(0xffffffffu, m_b, off));
         if (m_b > m_run) {
-            const float c = exp2f(m_run - m_b);     // 0 on the first batch
-            l *= c; lv *= c; o *= c;
+            const float c = exp2f(m_run - m_b);         // 0 on the first batch
+            l *= c; lv *= c;
+            o.x *= c; o.y *= c; o.z *= c; o.w *= c;
             m_run = m_b;
         }
+        const float w_mine = st.y > 0.f ? exp2f(st.x - m_run) : 0.f;
 #pragma unroll
         for (int u = 0; u < kCombineBatch; ++u) {
             if (u < n) {
-                const float4 st = stat_s[u];
-                if (st.y > 0.f) {
-                    const float w = exp2f(st.x - m_run);
-                    l = fmaf(w, st.y, l);
-                    lv = fmaf(w, st.z, lv);
-                    o = fmaf(w, v[u], o);
-                }
+                const float w = __shfl_sync(0xffffffffu, w_mine, u);
+                const float lu = __shfl_sync(0xffffffffu, st.y, u);
+                const float lvu = __shfl_sync(0xffffffffu, st.z, u);
+                l = fmaf(w, lu, l);
+                lv = fmaf(w, lvu, lv);
+                o.x = fmaf(w, v[u].x, o.x);
+                o.y = fmaf(w, v[u].y, o.y);
+                o.z = fmaf(w, v[u].z, o.z);
+                o.w = fmaf(w, v[u].w, o.w);
             }
         }
     }
     const float inv = 1.f / l;
     const int g = r / p.G, hg = r - g * p.G;
     const size_t row = ((size_t)b * p.gamma + g) * p.Hq + kvh * p.G + hg;
-    if (d < D) reinterpret_cast<__nv_bfloat16 *>(p.out)[row * D + d] = __float2bfloat16_rn(o * inv);
-    if (d == 0) p.mass[row] = lv * inv;
+    if (active) {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(o.x * inv, o.y * inv);
+        __nv_bfloat162 hi = __floats2bfloat162_rn(o.z * inv, o.w * inv);
+        uint2 pk;
+        pk.x = *reinterpret_cast<uint32_t *>(&lo);
+        pk.y = *reinterpret_cast<uint32_t *>(&hi);
+        *reinterpret_cast<uint2 *>(p.out + row * D + lane * 4) = pk;
+    }
+    if (lane == 0) p.mass[row] = lv * inv;
 }
 
 }  // namespace
@@ -286,14 +299,14 @@ cudaError_t launch_attn_simt(const AttnParams &p, const SeqInfo &seq, cudaStream
 cudaError_t launch_attn_combine(const AttnParams &p, cudaStream_t stream, int *launches)
 {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.M, p.Hkv, p.B);
-    cfg.blockDim = dim3(128, 1, 1);
+    cfg.gridDim = dim3((p.M + kCombineWarps - 1) / kCombineWarps, p.Hkv, p.B);
+    cfg.blockDim = dim3(32 * kCombineWarps, 1, 1);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 0;   // an early-launched combine grid piles up on the few idle SMs: plain launch
+    cfg.numAttrs = p.pdl ? 1 : 0;
     cudaError_t err = cudaLaunchKernelEx(&cfg, attn_combine_kernel, p);
     ++*launches;
     return err != cudaSuccess ? err : cudaGetLastError();

@@ -245,7 +245,6 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             mbar_init(drain_bar, 1);
             mbar_init(done_bar, kSoftmaxWarps + 1);
             mbar_fence_init();
-            grid_launch_dependents();
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -675,6 +674,10 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             bool all_done = false;
             for (int tries = 0; tries < 4 && !all_done; ++tries) all_done = wait_unconditional(done_bar, 0);
             if (*abort_flag || !all_done) atomicOr(p.status, LVSPEC_DEV_WAIT_EXPIRED);
+            // this CTA is done but for freeing TMEM: a dependent launch may be scheduled
+            // once every CTA has come this far (earlier, its CTAs would pile up on the
+            // few SMs this grid leaves idle)
+            grid_launch_dependents();
         }
         __syncwarp();
         tc_fence_after();
