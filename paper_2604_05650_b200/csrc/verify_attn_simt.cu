@@ -205,7 +205,7 @@ attn_simt_kernel(const AttnParams p, const SeqInfo seq)
 // one round trip to L2.  The running reference exponent moves up between
 // batches like an online softmax.
 constexpr int kCombineBatch = 32;
-constexpr int kCombineWarps = 4;
+constexpr int kCombineWarps = 2;
 
 __global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const AttnParams p)
 {

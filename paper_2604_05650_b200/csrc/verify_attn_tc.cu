@@ -215,18 +215,29 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     // once; the other warps prepare shared memory and TMEM meanwhile.
     int first_k = 0, first_v = 0;   // loads issued before the CTA-wide barrier
     if (warp == 0) {
-        if (lane == 0) {
-            // the TMA unit fetches the descriptors while the barriers are set up
-            prefetch_tensormap(&tmap_k);
-            prefetch_tensormap(&tmap_v);
-            prefetch_tensormap(&tmap_q);
-            // first the barriers the loads complete on, so that the loads can go out
-            for (int s = 0; s < cfg.ks; ++s) mbar_init(k_full(s), 1);
-            for (int s = 0; s < cfg.vs; ++s) mbar_init(v_full(s), 1);
-            mbar_init(q_full, 1);
-            *abort_flag = 0;
+        // the TMA unit fetches the descriptors while the barriers are set up
+        if (lane == 0) prefetch_tensormap(&tmap_k);
+        if (lane == 1) prefetch_tensormap(&tmap_v);
+        if (lane == 2) prefetch_tensormap(&tmap_q);
+        {
+            // one barrier per lane, all at once (an mbarrier.init costs about a hundred
+            // cycles): barriers sit in the order k_full, k_empty, v_full, v_empty,
+            // s_full[2], s_free[2], p_full, p_free, drain, done, q_full
+            const int n_kv = 2 * cfg.ks + 2 * cfg.vs;
+            const int n_bars = n_kv + 4 + 2 * cfg.pb + 3;
+            if (lane < n_bars) {
+                const int j = lane - n_kv;       // index among the barriers after the rings
+                uint32_t count = 1;
+                if (j >= 2 && j < 4 + cfg.pb) count = kSoftmaxWarps;           // s_free, p_full
+                else if (j == 4 + 2 * cfg.pb + 1) count = kSoftmaxWarps + 1;   // done
+                mbar_init(bar0 + 8 * lane, count);
+            }
+            if (lane == 0) *abort_flag = 0;
             mbar_fence_init();
             fence_proxy_async_smem();
+        }
+        __syncwarp();
+        if (lane == 0) {
             // inputs may come from the kernel before this one in the stream
             grid_dependency_wait();
             mbar_arrive_expect_tx(q_full, (uint32_t)M * 256u);
@@ -238,13 +249,6 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 if (i < first_k) load_k(i);
                 load_v(i);
             }
-            for (int s = 0; s < cfg.ks; ++s) mbar_init(k_empty(s), 1);
-            for (int s = 0; s < cfg.vs; ++s) mbar_init(v_empty(s), 1);
-            for (int s = 0; s < 2; ++s) { mbar_init(s_full(s), 1); mbar_init(s_free(s), kSoftmaxWarps); }
-            for (int s = 0; s < cfg.pb; ++s) { mbar_init(p_full(s), kSoftmaxWarps); mbar_init(p_free(s), 1); }
-            mbar_init(drain_bar, 1);
-            mbar_init(done_bar, kSoftmaxWarps + 1);
-            mbar_fence_init();
         }
         __syncwarp();
     } else if (warp == 1) {
