@@ -197,17 +197,21 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     const uint32_t q_full = drain_bar + 16;
     const int bh = b * p.Hkv + kvh;
 
+    // the cache is read once per call: it should not push the split partials out of L2
+    const uint64_t stream_policy = l2_evict_first_policy();
     auto load_k = [&](int i) {
         const int ks = i % cfg.ks, pos0 = (t_begin + i) * kTilePos;
         mbar_arrive_expect_tx(k_full(ks), kSlotBytes);
-        tma_load_3d(base + sm.k + ks * kSlotBytes, &tmap_k, k_full(ks), 0, pos0, bh);
-        tma_load_3d(base + sm.k + ks * kSlotBytes + kBoxBytes, &tmap_k, k_full(ks), 64, pos0, bh);
+        tma_load_3d_hint(base + sm.k + ks * kSlotBytes, &tmap_k, k_full(ks), 0, pos0, bh, stream_policy);
+        tma_load_3d_hint(base + sm.k + ks * kSlotBytes + kBoxBytes, &tmap_k, k_full(ks), 64, pos0, bh,
+                         stream_policy);
     };
     auto load_v = [&](int i) {
         const int vsl = i % cfg.vs, pos0 = (t_begin + i) * kTilePos;
         mbar_arrive_expect_tx(v_full(vsl), kSlotBytes);
-        tma_load_3d(base + sm.v + vsl * kSlotBytes, &tmap_v, v_full(vsl), 0, pos0, bh);
-        tma_load_3d(base + sm.v + vsl * kSlotBytes + kBoxBytes, &tmap_v, v_full(vsl), 64, pos0, bh);
+        tma_load_3d_hint(base + sm.v + vsl * kSlotBytes, &tmap_v, v_full(vsl), 0, pos0, bh, stream_policy);
+        tma_load_3d_hint(base + sm.v + vsl * kSlotBytes + kBoxBytes, &tmap_v, v_full(vsl), 64, pos0, bh,
+                         stream_policy);
     };
 
     // ------------------------------------------------------------------ prologue
