@@ -362,10 +362,15 @@ def run_ours(args, cfg):
         peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
     else:
         peak, peak_src = 6650.0, "fallback"
+    # DRAM bytes per launch from the committed ncu capture; null once the kernel has changed
     traffic = None
     tr_path = os.path.join(ROOT, "profiles", "traffic.json")
     if os.path.exists(tr_path):
-        traffic = json.load(open(tr_path)).get(f"config{cfg_id_of(cfg)}")
+        import hashlib
+        tr = json.load(open(tr_path))
+        src = os.path.join(ROOT, tr.get("kernel_source", ""))
+        if os.path.exists(src) and hashlib.sha256(open(src, "rb").read()).hexdigest() == tr.get("kernel_source_sha256"):
+            traffic = tr.get(f"config{cfg_id_of(cfg)}")
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "peak_source": peak_src, "kernel": "verify attention (one layer)",
                 "us_per_launch": us_per_launch, "bytes_per_launch": bytes_per_launch,
