@@ -219,6 +219,22 @@ def cfg_id_of(cfg):
 # --------------------------------------------------------------------------- #
 # our arm
 # --------------------------------------------------------------------------- #
+def slowest_rank_ms(ms_local, world, dist, device):
+    """Replicas only: every rank runs the same workload on its own GPU; the job
+    takes as long as its slowest rank (MAX over ranks of the device-timed ms)."""
+    import torch
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(world, batch, gamma, ms_step):
+    """Verified draft tokens per second of the whole job: all ranks' tokens over
+    the slowest rank's step time."""
+    return world * batch * gamma / (ms_step * 1e-3)
+
+
 def device_workload(cfg, dev, torch):
     """Synthetic inputs of the config's recipe drawn on the device (seeded):
     Q, K, V ~ N(0,1) in bf16 with the +0.5 shift of visual keys on 8 coordinates
@@ -345,12 +361,9 @@ def run_ours(args, cfg):
     status = ctx.device_status()
     ms_total = ev0.elapsed_time(ev1)
     ms_attn = sum(a.elapsed_time(b) for a, b in attn_ev) / args.steps
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total_max = float(t.item())
+    ms_total_max = slowest_rank_ms(ms_total, world, dist, dev)
     ms_step = ms_total_max / args.steps
-    value = world * B * g / (ms_step * 1e-3)
+    value = whole_job_tokens_per_s(world, B, g, ms_step)
     accepted = int(alen.sum().item())
 
     # roofline of the dominant kernel: one verification-attention launch
@@ -434,14 +447,11 @@ def run_e2e(args, cfg, ctx, stream, qs, ks, vs_, logits, draft, torch, dev, worl
     stream.synchronize()
     barrier()
     ms = ev0.elapsed_time(ev1) / steps
-    t = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms = float(t.item())
+    ms = slowest_rank_ms(ms, world, dist, dev)
     h2d = cfg.layers * (hq[0].numel() * 2 + 2 * hk[0].numel() * 2) + hlog.numel() * 4 + hdraft.numel() * 4 \
         + hmass.numel() * 4
     d2h = cfg.layers * (hout.numel() * 2 + hmass.numel() * 4) + hlen.numel() * 4
-    return {"value": world * B * g / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+    return {"value": whole_job_tokens_per_s(world, B, g, ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": ms, "steps": steps,
             "note": "K/V caches of every layer cross PCIe each step"}
 

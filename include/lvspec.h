@@ -89,7 +89,11 @@ typedef struct {
  * the calling thread during each call).  Allocates the scratch memory the
  * kernels need (a few MiB, grown on demand by later calls) and zeroes it.
  * Errors: INVALID_ARG (null out pointer, bad ordinal), CUDA (no device or
- * driver), WORKSPACE. */
+ * driver), WORKSPACE.
+ * The attention kernels of a context are launched "programmatically dependent"
+ * on the kernel before them in the stream (their set-up overlaps that kernel's
+ * tail; they still wait for it to finish before they read any input).  The
+ * environment variable LVSPEC_NO_PDL=1, read here, makes them plain launches. */
 lvspec_status_t lvspec_create(lvspec_ctx_t **ctx, int device);
 
 /* Synchronises the context's stream, frees its scratch memory and the context. */

@@ -213,3 +213,26 @@ def test_sweep_point_single_split(ctx, oracle_mod, kernel):
     tensor-core kernel then normalises and writes the results itself."""
     cfg = W.sweep_config(gamma=4, kv_len=4096, batch=16, point=9)
     _check(ctx, oracle_mod, W.attention_inputs(cfg), kernel=kernel)
+
+
+def test_plain_launches_give_the_same_results(oracle_mod, monkeypatch):
+    """LVSPEC_NO_PDL=1 (read when the context is created) launches the attention
+    kernels without programmatic dependence; results must not depend on it."""
+    from paper_2604_05650_b200 import binding
+    from gpu_util import run_attention
+    case = _case(21, 2, 8, 10, 2, 128, 1500, [1500, 777], [[100, 1200], [0, 700]])
+    outs = []
+    for flag in ("1", "0"):
+        monkeypatch.setenv("LVSPEC_NO_PDL", flag)
+        c = binding.Context(0)
+        try:
+            # several calls back to back, so that launches do follow one another
+            for _ in range(3):
+                res = run_attention(c, *case, kernel=2)
+            outs.append(res)
+        finally:
+            c.close()
+    assert (outs[0][0] == outs[1][0]).all() and (outs[0][1] == outs[1][1]).all()
+    ref_out, ref_mass = oracle_mod.verify_attention(*case)
+    from gpu_util import assert_attention_close
+    assert_attention_close(outs[0][0], outs[0][1], ref_out, ref_mass)
