@@ -193,3 +193,64 @@ int lvspec_oracle_n_loose(double lambda, int gamma)
 {
     return (int)floor(lambda * (double)gamma + 1e-9);
 }
+
+/*
+ * Visual relevance of the draft tokens as the paper defines it (Sec. 3.1,
+ * Eq. 4): the cosine similarity between the final-layer hidden state of each
+ * draft token and that of every visual token, then the mean of the N largest
+ * similarities along the visual dimension.
+ *
+ *   h_draft   bf16 bits [B, K, d]     H_D^s of Eq. 3
+ *   h_visual  bf16 bits [B, lv, d]    H_V of Eq. 3
+ *   top_n     N of Eq. 4 (the paper runs N = 10); min(N, lv) values are averaged
+ *   relevance fp64 [B, K]             A_s
+ *   cosines   optional fp64 [B, K, lv]
+ *
+ * A zero vector has no direction: its cosine with anything is taken as 0 (the
+ * paper does not meet the case).
+ */
+static int cmp_desc(const void *a, const void *b)
+{
+    const double x = *(const double *)a, y = *(const double *)b;
+    return (x < y) - (x > y);
+}
+
+void lvspec_oracle_visual_relevance(const uint16_t *h_draft, const uint16_t *h_visual,
+                                    int B, int K, int lv, int d, int top_n,
+                                    double *relevance, double *cosines)
+{
+    const long units = (long)B * K;
+#pragma omp parallel
+    {
+        double *c = (double *)malloc(sizeof(double) * (size_t)(lv > 0 ? lv : 1));
+        double *hd = (double *)malloc(sizeof(double) * (size_t)d);
+#pragma omp for schedule(dynamic, 1)
+        for (long u = 0; u < units; ++u) {
+            const int b = (int)(u / K), k = (int)(u % K);
+            const uint16_t *drow = h_draft + ((size_t)b * K + k) * d;
+            double nd = 0.0;
+            for (int t = 0; t < d; ++t) { hd[t] = bf16_to_double(drow[t]); nd += hd[t] * hd[t]; }
+            nd = sqrt(nd);
+            for (int j = 0; j < lv; ++j) {
+                const uint16_t *vrow = h_visual + ((size_t)b * lv + j) * d;
+                double dot = 0.0, nv = 0.0;
+                for (int t = 0; t < d; ++t) {
+                    const double x = bf16_to_double(vrow[t]);
+                    dot += hd[t] * x;
+                    nv += x * x;
+                }
+                nv = sqrt(nv);
+                c[j] = (nd > 0.0 && nv > 0.0) ? dot / (nd * nv) : 0.0;
+                if (cosines) cosines[((size_t)b * K + k) * (size_t)lv + j] = c[j];
+            }
+            qsort(c, (size_t)lv, sizeof(double), cmp_desc);
+            const int n = top_n < lv ? top_n : lv;
+            double sum = 0.0;
+            for (int j = 0; j < n; ++j) sum += c[j];
+            relevance[(size_t)b * K + k] = n > 0 ? sum / n : 0.0;
+        }
+        free(c);
+        free(hd);
+    }
+}
+

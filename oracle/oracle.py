@@ -43,6 +43,8 @@ def _load():
         lib.lvspec_oracle_verify_attention.restype = None
         lib.lvspec_oracle_loose_accept.argtypes = [p, p, p, i, i, i, i, i, i, p, p, p]
         lib.lvspec_oracle_loose_accept.restype = None
+        lib.lvspec_oracle_visual_relevance.argtypes = [p, p, i, i, i, i, i, p, p]
+        lib.lvspec_oracle_visual_relevance.restype = None
         lib.lvspec_oracle_n_loose.argtypes = [ctypes.c_double, i]
         lib.lvspec_oracle_n_loose.restype = i
         try:
@@ -115,3 +117,19 @@ def loose_accept(logits, draft, mass, n_loose: int, window: int):
 
 def n_loose(lam: float, gamma: int) -> int:
     return int(_load().lvspec_oracle_n_loose(float(lam), int(gamma)))
+
+
+def visual_relevance(h_draft, h_visual, top_n: int, return_cosines: bool = False):
+    """h_draft [B,K,d], h_visual [B,lv,d] as uint16 bf16 bit patterns.  Returns the
+    paper's relevance score A_s, fp64 [B,K] (and the cosines [B,K,lv])."""
+    lib = _load()
+    h_draft = np.ascontiguousarray(h_draft, dtype=np.uint16)
+    h_visual = np.ascontiguousarray(h_visual, dtype=np.uint16)
+    B, K, d = h_draft.shape
+    Bv, lv, dv = h_visual.shape
+    assert (Bv, dv) == (B, d)
+    rel = np.empty((B, K), dtype=np.float64)
+    cos = np.empty((B, K, lv), dtype=np.float64) if return_cosines else None
+    lib.lvspec_oracle_visual_relevance(_ptr(h_draft), _ptr(h_visual), B, K, lv, d, int(top_n),
+                                       _ptr(rel), _ptr(cos))
+    return (rel, cos) if return_cosines else rel

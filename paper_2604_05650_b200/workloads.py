@@ -170,3 +170,35 @@ def synthetic_mass(cfg: VerifyConfig, batch: int | None = None) -> np.ndarray:
     B = cfg.batch if batch is None else batch
     rng = np.random.default_rng([cfg.seed, 0x3A55])
     return rng.random((B, cfg.gamma, cfg.n_q_heads), dtype=np.float32)
+
+
+# ----------------------------------------------------------------------------
+# hidden states for the paper's own relevance score (Eq. 4)
+# ----------------------------------------------------------------------------
+def relevance_inputs(cfg: VerifyConfig, n_visual: int | None = None, dim: int | None = None,
+                     batch: int | None = None):
+    """Synthetic final-layer hidden states (the trained models are not available).
+
+    h_draft   uint16 [B, gamma, d]   bf16 bits, H_D of Eq. 3
+    h_visual  uint16 [B, lv, d]      bf16 bits, H_V of Eq. 3
+
+    d defaults to n_q_heads * head_dim and lv to the config's visual span.  Rows
+    ~ N(0, 1); every other draft row is pulled towards a small random set of
+    "salient" visual rows (weight 0.6), so that its largest similarities stand
+    out from the background the way Sec. 3.1 describes for visual-relevant
+    tokens; the remaining draft rows stay unrelated to the video.
+    """
+    B = cfg.batch if batch is None else batch
+    lv = cfg.span[1] - cfg.span[0] if n_visual is None else int(n_visual)
+    d = cfg.n_q_heads * cfg.head_dim if dim is None else int(dim)
+    g = cfg.gamma
+    rng = np.random.default_rng([cfg.seed, 0x4E1])
+    hv = rng.standard_normal((B, lv, d), dtype=np.float32)
+    hd = rng.standard_normal((B, g, d), dtype=np.float32)
+    for b in range(B):
+        for k in range(0, g, 2):
+            n_sal = int(rng.integers(1, 13))
+            rows = rng.choice(lv, size=min(n_sal, lv), replace=False)
+            hd[b, k] = np.float32(0.8) * hd[b, k] + np.float32(0.6) * hv[b, rows].mean(axis=0) * \
+                np.float32(np.sqrt(len(rows)))
+    return f32_to_bf16_bits(hd), f32_to_bf16_bits(hv)
