@@ -224,6 +224,41 @@ lvspec_status_t lvspec_loose_accept_host(lvspec_ctx_t *ctx, int32_t batch, int32
                                          const lvspec_thresholds_t *thresholds,
                                          int32_t shift_window, int32_t *accept_len);
 
+/* ---- the paper's own relevance score -------------------------------------------
+ *
+ * Sec. 3.1, Eq. 4: the visual relevance A_s of draft token k is the mean of the
+ * N largest cosine similarities between its final-layer hidden state H_D[k] and
+ * the final-layer hidden states H_V[j] of the visual tokens (Eq. 3; the paper
+ * runs N = 10).  The result feeds lvspec_loose_accept as `visual_mass` with
+ * n_mass_heads = 1, in place of the attention's visual mass.
+ *
+ * H_V is fixed after prefill, so the reciprocal norms of its rows are computed
+ * once (lvspec_row_inv_norms) and passed to every step's call.
+ *
+ *   lvspec_row_inv_norms:
+ *     x         device, bf16  [rows, dim]     dim a multiple of 8
+ *     inv_norm  device, fp32  [rows]          (written) 1 / ||x_r||, 0 for a zero row
+ *
+ *   lvspec_visual_relevance:
+ *     h_draft          device, bf16  [B, gamma, dim]       H_D of this step
+ *     h_visual         device, bf16  [B, n_visual, dim]    H_V
+ *     visual_inv_norm  device, fp32  [B, n_visual]         from lvspec_row_inv_norms
+ *     top_n            N >= 1; min(N, n_visual) similarities are averaged
+ *     relevance        device, fp32  [B, gamma]            (written) A_s
+ *
+ * A zero vector has cosine 0 with everything.  Dot products are bf16 x bf16
+ * accumulated in fp32 on the tensor cores; norms, cosines and the Top-N mean are
+ * fp32.  dim must be a multiple of 64, n_visual >= 1, gamma <= LVSPEC_MAX_GAMMA.
+ * Errors: INVALID_ARG (null or misaligned pointers, sizes out of range),
+ * UNSUPPORTED (dim not a multiple of 64), WORKSPACE / CUDA.
+ */
+lvspec_status_t lvspec_row_inv_norms(lvspec_ctx_t *ctx, int64_t rows, int32_t dim, const void *x,
+                                     float *inv_norm);
+lvspec_status_t lvspec_visual_relevance(lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,
+                                        int32_t n_visual, int32_t dim, const void *h_draft,
+                                        const void *h_visual, const float *visual_inv_norm,
+                                        int32_t top_n, float *relevance);
+
 /* ---- loose acceptance without any allocation ---------------------------------
  *
  * The paper has no counterpart of this call: it is the operation of

@@ -28,7 +28,7 @@ EXPORTS = (
     "lvspec_last_error", "lvspec_status_string", "lvspec_launch_count",
     "lvspec_attention_splits", "lvspec_verify_attention", "lvspec_verify_attention_host",
     "lvspec_loose_accept", "lvspec_loose_accept_ex", "lvspec_loose_accept_host",
-    "lvspec_loose_accept_static",
+    "lvspec_loose_accept_static", "lvspec_row_inv_norms", "lvspec_visual_relevance",
 )
 
 
@@ -82,6 +82,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lvspec_loose_accept.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp]
     lib.lvspec_loose_accept_ex.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp, vp, vp]
     lib.lvspec_loose_accept_host.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp]
+    lib.lvspec_row_inv_norms.argtypes = [vp, ctypes.c_int64, i32, vp, vp]
+    lib.lvspec_visual_relevance.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, i32, vp]
     lib.lvspec_loose_accept_static.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp,
                                                ctypes.c_char_p, ctypes.c_size_t]
     for name in EXPORTS:
@@ -179,6 +181,16 @@ class Context:
             self._h, batch, gamma, vocab, n_mass_heads, _addr(target_logits),
             _addr(draft_tokens), _addr(visual_mass), ctypes.byref(th), int(shift_window),
             _addr(accept_len), _addr(target_tokens), _addr(accepted)))
+
+    # -- the paper's own relevance score (Eq. 4) ---------------------------------
+    def row_inv_norms(self, rows, dim, x, inv_norm) -> None:
+        self._check(self._lib.lvspec_row_inv_norms(self._h, int(rows), int(dim), _addr(x), _addr(inv_norm)))
+
+    def visual_relevance(self, batch, gamma, n_visual, dim, h_draft, h_visual, visual_inv_norm,
+                         top_n, relevance) -> None:
+        self._check(self._lib.lvspec_visual_relevance(
+            self._h, batch, gamma, n_visual, dim, _addr(h_draft), _addr(h_visual),
+            _addr(visual_inv_norm), int(top_n), _addr(relevance)))
 
     def loose_accept_host(self, batch, gamma, vocab, n_mass_heads, target_logits, draft_tokens,
                           visual_mass, accept_len, shift_window, lam: float = 0.7,

@@ -449,6 +449,72 @@ lvspec_status_t lvspec_verify_attention_host(lvspec_ctx_t *ctx, const lvspec_att
     return LVSPEC_OK;
 }
 
+lvspec_status_t lvspec_row_inv_norms(lvspec_ctx_t *ctx, int64_t rows, int32_t dim, const void *x,
+                                     float *inv_norm)
+{
+    if (!ctx) return LVSPEC_ERR_INVALID_ARG;
+    if (!x || !inv_norm) return fail(ctx, LVSPEC_ERR_INVALID_ARG, "null argument");
+    if (rows < 1 || rows > (int64_t(1) << 31) * 8 - 8)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "rows out of range");
+    if (dim < 8 || dim % 8 != 0) return fail(ctx, LVSPEC_ERR_INVALID_ARG, "dim must be a positive multiple of 8");
+    if (!aligned16(x) || (reinterpret_cast<uintptr_t>(inv_norm) & 3u))
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "misaligned device pointer");
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
+    int launches = 0;
+    e = launch_row_inv_norms(static_cast<const uint16_t *>(x), rows, dim, inv_norm, ctx->stream, &launches);
+    ctx->launches += launches;
+    if (e != cudaSuccess) return cuda_fail(ctx, "norm kernel launch", e);
+    return LVSPEC_OK;
+}
+
+lvspec_status_t lvspec_visual_relevance(lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,
+                                        int32_t n_visual, int32_t dim, const void *h_draft,
+                                        const void *h_visual, const float *visual_inv_norm,
+                                        int32_t top_n, float *relevance)
+{
+    if (!ctx) return LVSPEC_ERR_INVALID_ARG;
+    if (!h_draft || !h_visual || !visual_inv_norm || !relevance)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "null argument");
+    if (batch < 1 || batch > LVSPEC_MAX_BATCH)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "batch outside 1..LVSPEC_MAX_BATCH");
+    if (gamma < 1 || gamma > LVSPEC_MAX_GAMMA)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "gamma outside 1..LVSPEC_MAX_GAMMA");
+    if (n_visual < 1 || (long long)batch * ((n_visual + 15) / 16) > 0x7fffffffLL)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "n_visual out of range");
+    if (top_n < 1) return fail(ctx, LVSPEC_ERR_INVALID_ARG, "top_n < 1");
+    if (dim < 64) return fail(ctx, LVSPEC_ERR_INVALID_ARG, "dim < 64");
+    if (dim % 64 != 0) return fail(ctx, LVSPEC_ERR_UNSUPPORTED, "dim must be a multiple of 64");
+    if (!aligned16(h_draft) || !aligned16(h_visual) ||
+        (reinterpret_cast<uintptr_t>(visual_inv_norm) & 3u) || (reinterpret_cast<uintptr_t>(relevance) & 3u))
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "misaligned device pointer");
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
+    lvspec_status_t st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes,
+                                relevance_scratch_bytes(batch, gamma, n_visual, dim), false);
+    if (st != LVSPEC_OK) return st;
+    RelevanceParams p;
+    std::memset(&p, 0, sizeof p);
+    p.h_draft = static_cast<const uint16_t *>(h_draft);
+    p.h_visual = static_cast<const uint16_t *>(h_visual);
+    p.v_inv_norm = visual_inv_norm;
+    p.cos_t = static_cast<float *>(ctx->scratch);
+    p.relevance = relevance;
+    p.status = ctx->status;
+    p.B = batch;
+    p.K = gamma;
+    p.lv = n_visual;
+    p.d = dim;
+    p.top_n = top_n;
+    p.lv_pad = (n_visual + 3) & ~3;
+    p.n_sm = ctx->n_sm;
+    int launches = 0;
+    e = launch_visual_relevance(p, ctx->stream, &launches);
+    ctx->launches += launches;
+    if (e != cudaSuccess) return cuda_fail(ctx, "relevance kernel launch", e);
+    return LVSPEC_OK;
+}
+
 lvspec_status_t lvspec_loose_accept_ex(lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,
                                        int32_t vocab, int32_t n_mass_heads,
                                        const float *target_logits, const int32_t *draft_tokens,

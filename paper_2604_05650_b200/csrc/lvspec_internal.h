@@ -61,4 +61,20 @@ struct AcceptParams {
 };
 cudaError_t launch_loose_accept(const AcceptParams &p, cudaStream_t stream, int *launches);
 
+struct RelevanceParams {
+    const uint16_t *h_draft;    // [B, K, d] bf16
+    const uint16_t *h_visual;   // [B, lv, d] bf16
+    const float *v_inv_norm;    // [B, lv]
+    float *cos_t;               // scratch [B, K, lv_pad]: cosines, one contiguous row per draft token
+    float *relevance;           // [B, K]
+    uint32_t *status;
+    int32_t B, K, lv, d, top_n;
+    int32_t lv_pad;             // lv rounded up to a multiple of 4
+    int32_t n_sm;
+};
+cudaError_t launch_row_inv_norms(const uint16_t *x, long long rows, int dim, float *out,
+                                 cudaStream_t stream, int *launches);
+cudaError_t launch_visual_relevance(const RelevanceParams &p, cudaStream_t stream, int *launches);
+size_t relevance_scratch_bytes(int B, int K, int lv, int d);
+
 }  // namespace lvspec

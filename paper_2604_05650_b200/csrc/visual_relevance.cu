@@ -1,0 +1,476 @@
+// The paper's own visual-relevance score (Sec. 3.1, Eq. 4): for every draft
+// token the mean of the N largest cosine similarities between its final-layer
+// hidden state and the visual tokens' final-layer hidden states.
+//
+// Three kernels per call:
+//   draft_prep_kernel   copies H_D into a row-padded scratch tile (rows padded to
+//                       a multiple of 16 with zeros) and takes its reciprocal norms
+//   cos_tc_kernel       streams H_V once (the HBM-bound part): per chunk of up to
+//                       128 visual rows, S[row, k] = H_V[row, :] . H_D[k, :] on the
+//                       tensor core (tcgen05, MMA M = 128 rows, N = padded K, the
+//                       hidden dimension in TMA stages of 64 channels), then
+//                       cosine = S * inv_norm_v[row] * inv_norm_d[k] to scratch
+//   topn_mean_kernel    exact Top-N mean per draft token by radix selection
+// The reciprocal norms of H_V's rows come from row_inv_norms_kernel, run once
+// after prefill.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "lvspec_internal.h"
+#include "sm100_ptx.cuh"
+
+namespace lvspec {
+namespace {
+
+using namespace ptx;
+
+// ------------------------------------------------------------------ row norms
+constexpr int kNormWarps = 8;
+
+__device__ __forceinline__ float sumsq_bf16x8(uint4 w, float acc)
+{
+    const uint32_t x[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float lo = __uint_as_float(x[i] << 16), hi = __uint_as_float(x[i] & 0xffff0000u);
+        acc = fmaf(lo, lo, acc);
+        acc = fmaf(hi, hi, acc);
+    }
+    return acc;
+}
+
+// one warp per row; dim a multiple of 8
+__global__ void __launch_bounds__(32 * kNormWarps)
+row_inv_norms_kernel(const uint16_t *x, long long rows, int dim, float *out)
+{
+    const long long r = (long long)blockIdx.x * kNormWarps + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    const uint4 *src = reinterpret_cast<const uint4 *>(x + r * dim);
+    float acc = 0.f;
+    for (int i = lane; i < dim / 8; i += 32) acc = sumsq_bf16x8(__ldg(src + i), acc);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) out[r] = acc > 0.f ? 1.f / sqrtf(acc) : 0.f;
+}
+
+// H_D [B, K, d] -> hd_pad [B, NP, d] (rows >= K zero) and dinv [B, NP]; one warp per padded row
+__global__ void __launch_bounds__(32 * kNormWarps)
+draft_prep_kernel(const uint16_t *hd, int B, int K, int NP, int dim, uint16_t *hd_pad, float *dinv)
+{
+    const int r = blockIdx.x * kNormWarps + (threadIdx.x >> 5);   // padded row index over B * NP
+    const int lane = threadIdx.x & 31;
+    if (r >= B * NP) return;
+    const int b = r / NP, k = r - b * NP;
+    uint4 *dst = reinterpret_cast<uint4 *>(hd_pad + (size_t)r * dim);
+    if (k >= K) {
+        for (int i = lane; i < dim / 8; i += 32) dst[i] = make_uint4(0, 0, 0, 0);
+        if (lane == 0) dinv[r] = 0.f;
+        return;
+    }
+    const uint4 *src = reinterpret_cast<const uint4 *>(hd + ((size_t)b * K + k) * dim);
+    float acc = 0.f;
+    for (int i = lane; i < dim / 8; i += 32) {
+        const uint4 w = __ldg(src + i);
+        dst[i] = w;
+        acc = sumsq_bf16x8(w, acc);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) dinv[r] = acc > 0.f ? 1.f / sqrtf(acc) : 0.f;
+}
+
+// ------------------------------------------------------------- cosine kernel
+constexpr int kCosThreads = 192;            // warp 0 producer, warp 1 MMA, warps 2-5 epilogue
+constexpr uint32_t kGroupBytes = 2048;      // 16 rows x 64 channels bf16
+constexpr uint32_t kVStageBytes = 8 * kGroupBytes;   // 128 rows
+
+struct CosParams {
+    RelevanceParams r;
+    const float *dinv;      // [B, NP]
+    int NP;                 // K padded to a multiple of 16 (MMA N)
+    int n_stages;
+    int tmem_cols;
+    int n_grp;              // groups of 16 rows per batch element
+    int total_groups;       // B * n_grp
+};
+
+// The chunks (up to 8 groups of 16 rows of one batch element) of one CTA's share
+// of the row groups; producer, MMA issuer and epilogue walk them in step.
+struct ChunkWalk {
+    int gg, end, n_grp;
+    int b, row0, n_groups;   // the current chunk
+    __device__ bool next()
+    {
+        if (gg >= end) return false;
+        b = gg / n_grp;
+        const int g0 = gg - b * n_grp;
+        n_groups = min(8, min(n_grp - g0, end - gg));
+        row0 = g0 * 16;
+        gg += n_groups;
+        return true;
+    }
+};
+
+__device__ __forceinline__ bool wait_teardown(uint32_t bar, uint32_t parity)
+{
+    const uint64_t t0 = global_timer_ns();
+    while (!mbar_try_wait(bar, parity))
+        if (global_timer_ns() - t0 > 1000000000ull) return false;
+    return true;
+}
+
+__global__ void __launch_bounds__(kCosThreads, 1)
+cos_tc_kernel(const CosParams P, const __grid_constant__ CUtensorMap tmap_v,
+              const __grid_constant__ CUtensorMap tmap_d)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const RelevanceParams &p = P.r;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int NP = P.NP, S = P.n_stages, KC = p.d / 64;
+    const uint32_t stage_bytes = kVStageBytes + (uint32_t)NP * 128u;
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *gbase = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bar0 = base + S * stage_bytes;
+    auto full = [&](int s) { return bar0 + 8 * s; };
+    auto empty = [&](int s) { return bar0 + 8 * (S + s); };
+    auto acc_full = [&](int s) { return bar0 + 8 * (2 * S + s); };
+    auto acc_free = [&](int s) { return bar0 + 8 * (2 * S + 2 + s); };
+    const uint32_t done_bar = bar0 + 8 * (2 * S + 4);
+    const uint32_t drain_bar = bar0 + 8 * (2 * S + 5);
+    const uint32_t misc = bar0 + 8 * (2 * S + 6);
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gbase + (misc - base));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(gbase + (misc - base) + 4);
+
+    // this CTA's share of the row groups: equal shares, sizes differ by at most one
+    ChunkWalk walk;
+    {
+        const int n_cta = gridDim.x, c = blockIdx.x;
+        const int per = P.total_groups / n_cta, rem = P.total_groups - per * n_cta;
+        walk.gg = c * per + min(c, rem);
+        walk.end = walk.gg + per + (c < rem ? 1 : 0);
+        walk.n_grp = P.n_grp;
+    }
+
+    if (warp == 0) {
+        if (lane == 0) prefetch_tensormap(&tmap_v);
+        if (lane == 1) prefetch_tensormap(&tmap_d);
+        const int n_bars = 2 * S + 6;
+        for (int j = lane; j < n_bars; j += 32) {
+            uint32_t count = 1;
+            if (j >= 2 * S + 2 && j < 2 * S + 4) count = 4;   // acc_free: the epilogue warps
+            else if (j == 2 * S + 4) count = 4;               // done
+            mbar_init(bar0 + 8 * j, count);
+        }
+        if (lane == 0) *abort_flag = 0;
+        mbar_fence_init();
+        fence_proxy_async_smem();
+    } else if (warp == 1) {
+        tmem_alloc(misc, (uint32_t)P.tmem_cols);
+        tmem_relinquish();
+    }
+    // the padded draft tile comes from the kernel before this one
+    grid_dependency_wait();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const uint64_t stream_policy = l2_evict_first_policy();
+            int n = 0;                       // stages filled so far
+            bool ok = true;
+            while (ok && walk.next()) {
+                for (int kc = 0; kc < KC; ++kc, ++n) {
+                    const int s = n % S;
+                    if (n >= S && !mbar_wait(empty(s), ((n / S) - 1) & 1, abort_flag)) { ok = false; break; }
+                    const uint32_t dst = base + s * stage_bytes;
+                    mbar_arrive_expect_tx(full(s), (uint32_t)walk.n_groups * kGroupBytes + (uint32_t)NP * 128u);
+                    for (int g = 0; g < walk.n_groups; ++g)
+                        tma_load_3d_hint(dst + g * kGroupBytes, &tmap_v, full(s), kc * 64,
+                                         walk.row0 + g * 16, walk.b, stream_policy);
+                    tma_load_3d(dst + kVStageBytes, &tmap_d, full(s), kc * 64, 0, walk.b);
+                }
+            }
+            if (*abort_flag) {
+                // wait (bounded) for the copies still in flight before the CTA leaves
+                for (int j = max(0, n - S); j < n; ++j) wait_teardown(full(j % S), (j / S) & 1);
+            }
+        }
+    } else if (warp == 1) {
+        // -------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_bf16(128, NP, 0, 0);
+            int s = 0, chunk = 0;
+            uint32_t round = 0;
+            bool ok = true;
+            while (ok && walk.next()) {
+                const int buf = chunk & 1;
+                if (chunk >= 2 && !mbar_wait(acc_free(buf), ((chunk >> 1) - 1) & 1, abort_flag)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * NP;
+                for (int kc = 0; kc < KC; ++kc) {
+                    if (!mbar_wait(full(s), round & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a0 = base + s * stage_bytes;
+                    const uint64_t da = make_smem_desc(a0, 16, 1024, kSwizzle128B);
+                    const uint64_t db = make_smem_desc(a0 + kVStageBytes, 16, 1024, kSwizzle128B);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_f16_ss(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc,
+                                   (kc | kk) != 0 ? 1u : 0u);
+                    mma_commit(empty(s));
+                    if (++s == S) { s = 0; ++round; }
+                }
+                if (!ok) break;
+                mma_commit(acc_full(buf));
+                ++chunk;
+            }
+            mma_commit(drain_bar);         // this thread's MMAs have drained
+            wait_teardown(drain_bar, 0);
+        }
+    } else {
+        // ---------------------------------------------------------- epilogue warps
+        const int wq = warp & 3;
+        const int row = wq * 32 + lane;                    // TMEM lane = row inside the chunk
+        const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
+        int chunk = 0;
+        while (walk.next()) {
+            const int buf = chunk & 1;
+            mbar_wait(acc_full(buf), (chunk >> 1) & 1, abort_flag);
+            tc_fence_after();
+            const int j = walk.row0 + row;                 // visual row of this thread
+            const bool valid = row < walk.n_groups * 16 && j < p.lv;
+            const float vin = valid ? __ldg(p.v_inv_norm + (size_t)walk.b * p.lv + j) : 0.f;
+            const float *dinv = P.dinv + (size_t)walk.b * NP;
+            float *dst = p.cos_t + (size_t)walk.b * p.K * p.lv_pad + j;
+            for (int c8 = 0; c8 < NP / 8; ++c8) {
+                uint32_t r[8];
+                tmem_ld_x8(tmem_base + buf * NP + lane_addr + c8 * 8, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const int kk = c8 * 8 + k;
+                    if (valid && kk < p.K)
+                        dst[(size_t)kk * p.lv_pad] = __uint_as_float(r[k]) * vin * __ldg(dinv + kk);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_free(buf));
+            ++chunk;
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(done_bar);
+    }
+
+    __syncwarp();
+    if (warp == 1) {
+        if (lane == 0) {
+            bool all_done = false;
+            for (int tries = 0; tries < 4 && !all_done; ++tries) all_done = wait_teardown(done_bar, 0);
+            if (*abort_flag || !all_done) atomicOr(p.status, LVSPEC_DEV_WAIT_EXPIRED);
+            grid_launch_dependents();
+        }
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, (uint32_t)P.tmem_cols);
+    }
+}
+
+// ------------------------------------------------------------- Top-N mean
+constexpr int kTopThreads = 1024;
+
+// order-preserving map float -> unsigned (larger float, larger key)
+__device__ __forceinline__ uint32_t float_key(float v)
+{
+    const uint32_t u = __float_as_uint(v);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_float(uint32_t k)
+{
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+// One CTA per (draft token, batch element): the exact mean of the n = min(N, lv)
+// largest of lv cosines.  Radix selection, 8 bits per pass from the top, finds
+// the key T of the n-th largest value and how many copies of T belong to the
+// top n; then the values above T are summed in a fixed order (each thread its
+// own elements by index, then a fixed tree), so the result is reproducible.
+__global__ void __launch_bounds__(kTopThreads) topn_mean_kernel(const RelevanceParams p)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    __shared__ uint32_t hist[256];
+    __shared__ uint32_t sel_prefix, sel_need;
+    __shared__ float warp_sum[kTopThreads / 32];
+    const int k = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    const float *row = p.cos_t + ((size_t)b * p.K + k) * p.lv_pad;
+    const int lv = p.lv;
+    const uint32_t n = (uint32_t)min(p.top_n, lv);
+
+    uint32_t prefix = 0, mask = 0, need = n;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = tid; i < 256; i += kTopThreads) hist[i] = 0;
+        __syncthreads();
+        for (int j = tid; j < lv; j += kTopThreads) {
+            const uint32_t key = float_key(__ldcg(row + j));
+            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t above = 0;
+            int bin = 255;
+            for (; bin > 0; --bin) {
+                if (above + hist[bin] >= need) break;
+                above += hist[bin];
+            }
+            sel_prefix = prefix | ((uint32_t)bin << shift);
+            sel_need = need - above;       // how many of this bin still belong to the top n
+        }
+        __syncthreads();
+        prefix = sel_prefix;
+        need = sel_need;
+        mask |= 255u << shift;
+        __syncthreads();
+    }
+    // prefix = key of the n-th largest value; `need` copies of it are inside the top n
+    float acc = 0.f;
+    for (int j = tid; j < lv; j += kTopThreads) {
+        const float v = __ldcg(row + j);
+        if (float_key(v) > prefix) acc += v;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if ((tid & 31) == 0) warp_sum[tid >> 5] = acc;
+    __syncthreads();
+    if (tid < 32) {
+        float s = tid < kTopThreads / 32 ? warp_sum[tid] : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (tid == 0) p.relevance[(size_t)b * p.K + k] = (s + (float)need * key_float(prefix)) / (float)n;
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// [B][rows][d] bf16 as a 3-D tensor; boxes of 64 channels x box_rows rows, 128-byte swizzle
+bool make_rows_map(CUtensorMap *map, const void *ptr, int d, int rows, int B, int box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)rows, (cuuint64_t)B};
+    const cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)rows * d * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cudaError_t launch_row_inv_norms(const uint16_t *x, long long rows, int dim, float *out,
+                                 cudaStream_t stream, int *launches)
+{
+    const long long blocks = (rows + kNormWarps - 1) / kNormWarps;
+    row_inv_norms_kernel<<<(unsigned)blocks, 32 * kNormWarps, 0, stream>>>(x, rows, dim, out);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+// Scratch layout behind p.cos_t: cosines [B, K, lv_pad] fp32, then the padded draft
+// tile [B, NP, d] bf16 (1024-byte aligned), then its reciprocal norms [B, NP].
+size_t relevance_scratch_bytes(int B, int K, int lv, int d)
+{
+    const int NP = (K + 15) & ~15;
+    const int lv_pad = (lv + 3) & ~3;
+    size_t o = (size_t)B * K * lv_pad * sizeof(float);
+    o = (o + 1023) & ~size_t(1023);
+    o += (size_t)B * NP * d * 2;
+    o = (o + 1023) & ~size_t(1023);
+    o += (size_t)B * NP * sizeof(float);
+    return o;
+}
+
+cudaError_t launch_visual_relevance(const RelevanceParams &p, cudaStream_t stream, int *launches)
+{
+    const int NP = (p.K + 15) & ~15;
+    size_t o = (size_t)p.B * p.K * p.lv_pad * sizeof(float);
+    o = (o + 1023) & ~size_t(1023);
+    uint16_t *hd_pad = reinterpret_cast<uint16_t *>(reinterpret_cast<char *>(p.cos_t) + o);
+    o += (size_t)p.B * NP * p.d * 2;
+    o = (o + 1023) & ~size_t(1023);
+    float *dinv = reinterpret_cast<float *>(reinterpret_cast<char *>(p.cos_t) + o);
+
+    draft_prep_kernel<<<(p.B * NP + kNormWarps - 1) / kNormWarps, 32 * kNormWarps, 0, stream>>>(
+        p.h_draft, p.B, p.K, NP, p.d, hd_pad, dinv);
+    ++*launches;
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+
+    CosParams P;
+    P.r = p;
+    P.dinv = dinv;
+    P.NP = NP;
+    const uint32_t stage_bytes = kVStageBytes + (uint32_t)NP * 128u;
+    int S = (int)((232448u - 1024u - 512u) / stage_bytes);
+    if (S > 12) S = 12;
+    P.n_stages = S;
+    int cols = 32;
+    while (cols < 2 * NP) cols <<= 1;
+    P.tmem_cols = cols;
+    P.n_grp = (p.lv + 15) / 16;
+    P.total_groups = p.B * P.n_grp;
+    CUtensorMap mv, md;
+    if (!make_rows_map(&mv, p.h_visual, p.d, p.lv, p.B, 16) || !make_rows_map(&md, hd_pad, p.d, NP, p.B, NP))
+        return cudaErrorInvalidValue;
+    const size_t smem = (size_t)S * stage_bytes + 8 * (2 * S + 6) + 16 + 1024;
+    err = cudaFuncSetAttribute(cos_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(P.total_groups < p.n_sm ? P.total_groups : p.n_sm), 1, 1);
+    cfg.blockDim = dim3(kCosThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    err = cudaLaunchKernelEx(&cfg, cos_tc_kernel, P, mv, md);
+    ++*launches;
+    if (err != cudaSuccess) return err;
+
+    cudaLaunchConfig_t cfg2 = {};
+    cfg2.gridDim = dim3((unsigned)p.K, (unsigned)p.B, 1);
+    cfg2.blockDim = dim3(kTopThreads, 1, 1);
+    cfg2.stream = stream;
+    cfg2.attrs = attr;
+    cfg2.numAttrs = 1;
+    err = cudaLaunchKernelEx(&cfg2, topn_mean_kernel, p);
+    ++*launches;
+    return err != cudaSuccess ? err : cudaGetLastError();
+}
+
+}  // namespace lvspec
