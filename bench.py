@@ -44,6 +44,8 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch layer by layer, no CUDA graph")
+    ap.add_argument("--no-next-rows", action="store_true",
+                    help="skip the timing of the paper's own relevance score (not part of the step)")
     ap.add_argument("--sweep", action="store_true",
                     help="run the head-shape sweep (BASELINE config 4): gamma x KV length x batch, one layer "
                          "per point; the JSON line then carries the per-point table under \"sweep\"")
@@ -398,6 +400,9 @@ def run_ours(args, cfg):
             "gpu_launches": launches_per_step * args.steps, "device_status": status,
             "cuda_graph": graph_attn is not None, "roofline": roofline, "clocks": clocks.summary()}
 
+    if not args.no_next_rows and world == 1:
+        line["next_rows"] = {"visual_relevance": time_visual_relevance(cfg, ctx, stream, torch, dev, peak)}
+
     # end to end through the host-buffer entry points
     if not args.no_e2e:
         line["e2e"] = run_e2e(args, cfg, ctx, stream, qs, ks, vs_, logits, draft, torch, dev, world, barrier, dist)
@@ -411,6 +416,41 @@ def run_ours(args, cfg):
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def time_visual_relevance(cfg, ctx, stream, torch, dev, peak):
+    """The paper's own relevance score (Eq. 4) on the config's visual span and
+    hidden size, N = 10: not part of the verify step this benchmark times (the
+    step scores positions by the attention's visual mass), measured beside it.
+    HBM-bound on the one pass over H_V; two H_V copies alternate (each > L2)."""
+    B, g = cfg.batch, cfg.gamma
+    lv, d = cfg.span[1] - cfg.span[0], cfg.n_q_heads * cfg.head_dim
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(cfg.seed + 77)
+    hv = [torch.randn((B, lv, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16) for _ in range(2)]
+    hd = torch.randn((B, g, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    inv = [torch.empty((B, lv), dtype=torch.float32, device=dev) for _ in range(2)]
+    rel = torch.empty((B, g), dtype=torch.float32, device=dev)
+    with torch.cuda.stream(stream):
+        for c in range(2):
+            ctx.row_inv_norms(B * lv, d, hv[c], inv[c])
+        for c in range(2):
+            ctx.visual_relevance(B, g, lv, d, hd, hv[c], inv[c], 10, rel)
+    stream.synchronize()
+    reps = 10
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for _ in range(reps):
+            for c in range(2):
+                ctx.visual_relevance(B, g, lv, d, hd, hv[c], inv[c], 10, rel)
+        e1.record(stream)
+    stream.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / (2 * reps)
+    nbytes = B * lv * d * 2 + B * lv * 4
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return {"us_per_call": us, "n_visual": lv, "dim": d, "top_n": 10, "bytes_per_call": nbytes,
+            "achieved_gbs": gbs, "frac_of_peak": gbs / peak, "launches_per_call": 3}
 
 
 def run_e2e(args, cfg, ctx, stream, qs, ks, vs_, logits, draft, torch, dev, world, barrier, dist):

@@ -5,10 +5,12 @@
 // Three kernels per call:
 //   draft_prep_kernel   copies H_D into a row-padded scratch tile (rows padded to
 //                       a multiple of 16 with zeros) and takes its reciprocal norms
-//   cos_tc_kernel       streams H_V once (the HBM-bound part): per chunk of up to
-//                       128 visual rows, S[row, k] = H_V[row, :] . H_D[k, :] on the
-//                       tensor core (tcgen05, MMA M = 128 rows, N = padded K, the
-//                       hidden dimension in TMA stages of 64 channels), then
+//   cos_tc_kernel       streams H_V once (the HBM-bound part): every CTA takes an
+//                       equal share of the visual rows, in chunks of up to 256
+//                       rows = two row blocks with one accumulator each;
+//                       S[row, k] = H_V[row, :] . H_D[k, :] on the tensor core
+//                       (tcgen05, MMA M = 128 rows, N = padded K, the hidden
+//                       dimension in TMA stages of 64 channels), then
 //                       cosine = S * inv_norm_v[row] * inv_norm_d[k] to scratch
 //   topn_mean_kernel    exact Top-N mean per draft token by radix selection
 // The reciprocal norms of H_V's rows come from row_inv_norms_kernel, run once
@@ -83,19 +85,22 @@ draft_prep_kernel(const uint16_t *hd, int B, int K, int NP, int dim, uint16_t *h
 // ------------------------------------------------------------- cosine kernel
 constexpr int kCosThreads = 192;            // warp 0 producer, warp 1 MMA, warps 2-5 epilogue
 constexpr uint32_t kGroupBytes = 2048;      // 16 rows x 64 channels bf16
-constexpr uint32_t kVStageBytes = 8 * kGroupBytes;   // 128 rows
+constexpr uint32_t kBlockBytes = 8 * kGroupBytes;    // one row block: 128 rows
+constexpr int kChunkGroups = 16;            // groups of 16 rows per chunk
+constexpr int kMaxStages = 24;
+constexpr uint32_t kBarBytes = 1024;        // barriers and the TMEM slot, ahead of the stages
 
 struct CosParams {
     RelevanceParams r;
     const float *dinv;      // [B, NP]
     int NP;                 // K padded to a multiple of 16 (MMA N)
-    int n_stages;
+    int smem_bytes;         // dynamic shared memory of the launch (after 1024-byte alignment)
     int tmem_cols;
     int n_grp;              // groups of 16 rows per batch element
     int total_groups;       // B * n_grp
 };
 
-// The chunks (up to 8 groups of 16 rows of one batch element) of one CTA's share
+// The chunks (up to 16 groups of 16 rows of one batch element) of one CTA's share
 // of the row groups; producer, MMA issuer and epilogue walk them in step.
 struct ChunkWalk {
     int gg, end, n_grp;
@@ -105,7 +110,7 @@ struct ChunkWalk {
         if (gg >= end) return false;
         b = gg / n_grp;
         const int g0 = gg - b * n_grp;
-        n_groups = min(8, min(n_grp - g0, end - gg));
+        n_groups = min(kChunkGroups, min(n_grp - g0, end - gg));
         row0 = g0 * 16;
         gg += n_groups;
         return true;
@@ -122,26 +127,12 @@ __device__ __forceinline__ bool wait_teardown(uint32_t bar, uint32_t parity)
 
 __global__ void __launch_bounds__(kCosThreads, 1)
 cos_tc_kernel(const CosParams P, const __grid_constant__ CUtensorMap tmap_v,
-              const __grid_constant__ CUtensorMap tmap_d)
+              const __grid_constant__ CUtensorMap tmap_v128, const __grid_constant__ CUtensorMap tmap_d)
 {
     extern __shared__ uint8_t smem_raw[];
     const RelevanceParams &p = P.r;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int NP = P.NP, S = P.n_stages, KC = p.d / 64;
-    const uint32_t stage_bytes = kVStageBytes + (uint32_t)NP * 128u;
-
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t *gbase = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t bar0 = base + S * stage_bytes;
-    auto full = [&](int s) { return bar0 + 8 * s; };
-    auto empty = [&](int s) { return bar0 + 8 * (S + s); };
-    auto acc_full = [&](int s) { return bar0 + 8 * (2 * S + s); };
-    auto acc_free = [&](int s) { return bar0 + 8 * (2 * S + 2 + s); };
-    const uint32_t done_bar = bar0 + 8 * (2 * S + 4);
-    const uint32_t drain_bar = bar0 + 8 * (2 * S + 5);
-    const uint32_t misc = bar0 + 8 * (2 * S + 6);
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gbase + (misc - base));
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(gbase + (misc - base) + 4);
+    const int NP = P.NP, KC = p.d / 64;
 
     // this CTA's share of the row groups: equal shares, sizes differ by at most one
     ChunkWalk walk;
@@ -152,10 +143,37 @@ cos_tc_kernel(const CosParams P, const __grid_constant__ CUtensorMap tmap_v,
         walk.end = walk.gg + per + (c < rem ? 1 : 0);
         walk.n_grp = P.n_grp;
     }
+    // A stage holds 64 channels of the tallest chunk this CTA can meet (row block 0,
+    // then row block 1, then the draft tile); the fewer rows, the more stages fit,
+    // and bytes in flight, not stages, are what covers the memory latency.
+    const int cap = max(1, min(kChunkGroups, walk.end - walk.gg));
+    const uint32_t d_off = cap <= 8 ? (uint32_t)cap * kGroupBytes : kBlockBytes + (uint32_t)(cap - 8) * kGroupBytes;
+    const uint32_t stage_bytes = (d_off + (uint32_t)NP * 128u + 1023u) & ~1023u;
+    // An MMA always reads whole row blocks of 128 rows (rows a chunk does not have are
+    // junk lanes nobody looks at), so from the last stage's start one or two full
+    // blocks must still lie inside the allocation.
+    const uint32_t read_extent = cap > 8 ? 2 * kBlockBytes : kBlockBytes;
+    const int S = min(kMaxStages,
+                      1 + (int)(((uint32_t)P.smem_bytes - kBarBytes - max(read_extent, stage_bytes)) / stage_bytes));
+
+    const uint32_t base0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *gbase = smem_raw + (base0 - smem_u32(smem_raw));
+    const uint32_t bar0 = base0;
+    const uint32_t base = base0 + kBarBytes;          // first stage
+    auto full = [&](int s) { return bar0 + 8 * s; };
+    auto empty = [&](int s) { return bar0 + 8 * (S + s); };
+    auto acc_full = [&](int s) { return bar0 + 8 * (2 * S + s); };
+    auto acc_free = [&](int s) { return bar0 + 8 * (2 * S + 2 + s); };
+    const uint32_t done_bar = bar0 + 8 * (2 * S + 4);
+    const uint32_t drain_bar = bar0 + 8 * (2 * S + 5);
+    const uint32_t misc = bar0 + 8 * (2 * S + 6);
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gbase + (misc - base0));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(gbase + (misc - base0) + 4);
 
     if (warp == 0) {
         if (lane == 0) prefetch_tensormap(&tmap_v);
         if (lane == 1) prefetch_tensormap(&tmap_d);
+        if (lane == 2) prefetch_tensormap(&tmap_v128);
         const int n_bars = 2 * S + 6;
         for (int j = lane; j < n_bars; j += 32) {
             uint32_t count = 1;
@@ -189,10 +207,21 @@ cos_tc_kernel(const CosParams P, const __grid_constant__ CUtensorMap tmap_v,
                     if (n >= S && !mbar_wait(empty(s), ((n / S) - 1) & 1, abort_flag)) { ok = false; break; }
                     const uint32_t dst = base + s * stage_bytes;
                     mbar_arrive_expect_tx(full(s), (uint32_t)walk.n_groups * kGroupBytes + (uint32_t)NP * 128u);
-                    for (int g = 0; g < walk.n_groups; ++g)
+                    // a full row block in one box of 128 rows, the rest in boxes of 16
+                    int g = 0;
+                    if (walk.n_groups >= 8) {
+                        tma_load_3d_hint(dst, &tmap_v128, full(s), kc * 64, walk.row0, walk.b, stream_policy);
+                        g = 8;
+                    }
+                    if (walk.n_groups == 16) {
+                        tma_load_3d_hint(dst + kBlockBytes, &tmap_v128, full(s), kc * 64, walk.row0 + 128,
+                                         walk.b, stream_policy);
+                        g = 16;
+                    }
+                    for (; g < walk.n_groups; ++g)
                         tma_load_3d_hint(dst + g * kGroupBytes, &tmap_v, full(s), kc * 64,
                                          walk.row0 + g * 16, walk.b, stream_policy);
-                    tma_load_3d(dst + kVStageBytes, &tmap_d, full(s), kc * 64, 0, walk.b);
+                    tma_load_3d(dst + d_off, &tmap_d, full(s), kc * 64, 0, walk.b);
                 }
             }
             if (*abort_flag) {
@@ -211,17 +240,24 @@ cos_tc_kernel(const CosParams P, const __grid_constant__ CUtensorMap tmap_v,
                 const int buf = chunk & 1;
                 if (chunk >= 2 && !mbar_wait(acc_free(buf), ((chunk >> 1) - 1) & 1, abort_flag)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * NP;
+                const uint32_t d_tmem = tmem_base + buf * 2 * NP;
+                const bool two_blocks = walk.n_groups > 8;
                 for (int kc = 0; kc < KC; ++kc) {
                     if (!mbar_wait(full(s), round & 1, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a0 = base + s * stage_bytes;
                     const uint64_t da = make_smem_desc(a0, 16, 1024, kSwizzle128B);
-                    const uint64_t db = make_smem_desc(a0 + kVStageBytes, 16, 1024, kSwizzle128B);
+                    const uint64_t db = make_smem_desc(a0 + d_off, 16, 1024, kSwizzle128B);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
                         mma_f16_ss(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc,
                                    (kc | kk) != 0 ? 1u : 0u);
+                    if (two_blocks) {
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            mma_f16_ss(d_tmem + NP, da + (uint64_t)((kBlockBytes >> 4) + kk * 2),
+                                       db + (uint64_t)(kk * 2), idesc, (kc | kk) != 0 ? 1u : 0u);
+                    }
                     mma_commit(empty(s));
                     if (++s == S) { s = 0; ++round; }
                 }
@@ -242,20 +278,24 @@ cos_tc_kernel(const CosParams P, const __grid_constant__ CUtensorMap tmap_v,
             const int buf = chunk & 1;
             mbar_wait(acc_full(buf), (chunk >> 1) & 1, abort_flag);
             tc_fence_after();
-            const int j = walk.row0 + row;                 // visual row of this thread
-            const bool valid = row < walk.n_groups * 16 && j < p.lv;
-            const float vin = valid ? __ldg(p.v_inv_norm + (size_t)walk.b * p.lv + j) : 0.f;
             const float *dinv = P.dinv + (size_t)walk.b * NP;
-            float *dst = p.cos_t + (size_t)walk.b * p.K * p.lv_pad + j;
-            for (int c8 = 0; c8 < NP / 8; ++c8) {
-                uint32_t r[8];
-                tmem_ld_x8(tmem_base + buf * NP + lane_addr + c8 * 8, r);
-                tmem_wait_ld();
+            const int n_blocks = walk.n_groups > 8 ? 2 : 1;
+            for (int blk = 0; blk < n_blocks; ++blk) {
+                const int rc = blk * 128 + row;                // row inside the chunk
+                const int j = walk.row0 + rc;                  // visual row of this thread
+                const bool valid = rc < walk.n_groups * 16 && j < p.lv;
+                const float vin = valid ? __ldg(p.v_inv_norm + (size_t)walk.b * p.lv + j) : 0.f;
+                float *dst = p.cos_t + (size_t)walk.b * p.K * p.lv_pad + j;
+                for (int c8 = 0; c8 < NP / 8; ++c8) {
+                    uint32_t r[8];
+                    tmem_ld_x8(tmem_base + (buf * 2 + blk) * NP + lane_addr + c8 * 8, r);
+                    tmem_wait_ld();
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const int kk = c8 * 8 + k;
-                    if (valid && kk < p.K)
-                        dst[(size_t)kk * p.lv_pad] = __uint_as_float(r[k]) * vin * __ldg(dinv + kk);
+                    for (int k = 0; k < 8; ++k) {
+                        const int kk = c8 * 8 + k;
+                        if (valid && kk < p.K)
+                            dst[(size_t)kk * p.lv_pad] = __uint_as_float(r[k]) * vin * __ldg(dinv + kk);
+                    }
                 }
             }
             tc_fence_before();
@@ -296,21 +336,86 @@ __device__ __forceinline__ float key_float(uint32_t k)
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
+constexpr int kTopPerThread = 32;      // fast path: lv <= 32 * 1024
+constexpr int kTopCandidates = 2048;
+
+// descending bitonic sort of a power-of-two array of keys in shared memory
+__device__ void bitonic_sort_desc(uint32_t *a, int n, int tid)
+{
+    for (int size = 2; size <= n; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            __syncthreads();
+            for (int i = tid; i < n / 2; i += kTopThreads) {
+                const int lo = 2 * i - (i & (stride - 1));      // index with the `stride` bit clear
+                const int hi = lo + stride;
+                const bool descending = (lo & size) == 0;
+                const uint32_t x = a[lo], y = a[hi];
+                if ((x < y) == descending) { a[lo] = y; a[hi] = x; }
+            }
+        }
+    }
+    __syncthreads();
+}
+
 // One CTA per (draft token, batch element): the exact mean of the n = min(N, lv)
-// largest of lv cosines.  Radix selection, 8 bits per pass from the top, finds
-// the key T of the n-th largest value and how many copies of T belong to the
-// top n; then the values above T are summed in a fixed order (each thread its
-// own elements by index, then a fixed tree), so the result is reproducible.
+// largest of lv cosines, summed in descending order of value (reproducible).
+//
+// Fast path (lv <= 32768, n <= 1024): every thread keeps its strided elements in
+// registers and reports its largest; the n-th largest of these 1024 maxima is
+// a lower bound of the n-th largest element, so only the few elements at or
+// above it are collected and sorted.  If the candidates do not fit (the large
+// values all sit in few threads' strides) or the row is longer, the general
+// path finds the n-th largest key by radix selection, 8 bits per pass.
 __global__ void __launch_bounds__(kTopThreads) topn_mean_kernel(const RelevanceParams p)
 {
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    __shared__ uint32_t keys[kTopCandidates];
     __shared__ uint32_t hist[256];
-    __shared__ uint32_t sel_prefix, sel_need;
+    __shared__ uint32_t sel_prefix, sel_need, n_cand;
     __shared__ float warp_sum[kTopThreads / 32];
     const int k = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
     const float *row = p.cos_t + ((size_t)b * p.K + k) * p.lv_pad;
     const int lv = p.lv;
     const uint32_t n = (uint32_t)min(p.top_n, lv);
+    float *out = p.relevance + (size_t)b * p.K + k;
+
+    if (lv <= kTopPerThread * kTopThreads && n <= (uint32_t)kTopThreads) {
+        uint32_t mine[kTopPerThread];
+        uint32_t best = 0;                                  // below every real key
+#pragma unroll
+        for (int i = 0; i < kTopPerThread; ++i) {
+            const int j = tid + i * kTopThreads;
+            mine[i] = j < lv ? float_key(__ldcg(row + j)) : 0u;
+            best = max(best, mine[i]);
+        }
+        keys[tid] = best;
+        if (tid == 0) n_cand = 0;
+        bitonic_sort_desc(keys, kTopThreads, tid);
+        const uint32_t bound = keys[n - 1];                 // >= n elements are at or above it
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < kTopPerThread; ++i) {
+            if (mine[i] >= bound && mine[i] != 0u) {
+                const uint32_t slot = atomicAdd(&n_cand, 1u);
+                if (slot < (uint32_t)kTopCandidates) keys[slot] = mine[i];
+            }
+        }
+        __syncthreads();
+        const uint32_t c = n_cand;
+        if (c <= (uint32_t)kTopCandidates) {
+            int pow2 = 32;
+            while ((uint32_t)pow2 < c) pow2 <<= 1;
+            for (int i = c + tid; i < pow2; i += kTopThreads) keys[i] = 0u;
+            bitonic_sort_desc(keys, pow2, tid);
+            if (tid == 0) {
+                float sum = 0.f;
+                for (uint32_t i = 0; i < n; ++i) sum += key_float(keys[i]);
+                *out = sum / (float)n;
+            }
+            return;
+        }
+        __syncthreads();
+    }
 
     uint32_t prefix = 0, mask = 0, need = n;
     for (int shift = 24; shift >= 0; shift -= 8) {
@@ -348,10 +453,10 @@ __global__ void __launch_bounds__(kTopThreads) topn_mean_kernel(const RelevanceP
     if ((tid & 31) == 0) warp_sum[tid >> 5] = acc;
     __syncthreads();
     if (tid < 32) {
-        float s = tid < kTopThreads / 32 ? warp_sum[tid] : 0.f;
+        float s2 = tid < kTopThreads / 32 ? warp_sum[tid] : 0.f;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        if (tid == 0) p.relevance[(size_t)b * p.K + k] = (s + (float)need * key_float(prefix)) / (float)n;
+        for (int o = 16; o > 0; o >>= 1) s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+        if (tid == 0) *out = (s2 + (float)need * key_float(prefix)) / (float)n;
     }
 }
 
@@ -433,19 +538,19 @@ cudaError_t launch_visual_relevance(const RelevanceParams &p, cudaStream_t strea
     P.r = p;
     P.dinv = dinv;
     P.NP = NP;
-    const uint32_t stage_bytes = kVStageBytes + (uint32_t)NP * 128u;
-    int S = (int)((232448u - 1024u - 512u) / stage_bytes);
-    if (S > 12) S = 12;
-    P.n_stages = S;
+    P.smem_bytes = 232448 - 1024;      // everything an SM offers, less the alignment slack
     int cols = 32;
-    while (cols < 2 * NP) cols <<= 1;
+    while (cols < 4 * NP) cols <<= 1;
     P.tmem_cols = cols;
     P.n_grp = (p.lv + 15) / 16;
     P.total_groups = p.B * P.n_grp;
-    CUtensorMap mv, md;
-    if (!make_rows_map(&mv, p.h_visual, p.d, p.lv, p.B, 16) || !make_rows_map(&md, hd_pad, p.d, NP, p.B, NP))
+    CUtensorMap mv, mv128, md;
+    if (!make_rows_map(&mv, p.h_visual, p.d, p.lv, p.B, 16) ||
+        // (fewer than 128 rows never make a full row block: the wide map is then not used)
+        !make_rows_map(&mv128, p.h_visual, p.d, p.lv, p.B, p.lv >= 128 ? 128 : 16) ||
+        !make_rows_map(&md, hd_pad, p.d, NP, p.B, NP))
         return cudaErrorInvalidValue;
-    const size_t smem = (size_t)S * stage_bytes + 8 * (2 * S + 6) + 16 + 1024;
+    const size_t smem = (size_t)P.smem_bytes + 1024;
     err = cudaFuncSetAttribute(cos_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     cudaLaunchAttribute attr[1];
@@ -458,7 +563,7 @@ cudaError_t launch_visual_relevance(const RelevanceParams &p, cudaStream_t strea
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    err = cudaLaunchKernelEx(&cfg, cos_tc_kernel, P, mv, md);
+    err = cudaLaunchKernelEx(&cfg, cos_tc_kernel, P, mv, mv128, md);
     ++*launches;
     if (err != cudaSuccess) return err;
 
