@@ -56,30 +56,36 @@ row_inv_norms_kernel(const uint16_t *x, long long rows, int dim, float *out)
     if (lane == 0) out[r] = acc > 0.f ? 1.f / sqrtf(acc) : 0.f;
 }
 
-// H_D [B, K, d] -> hd_pad [B, NP, d] (rows >= K zero) and dinv [B, NP]; one warp per padded row
-__global__ void __launch_bounds__(32 * kNormWarps)
+// H_D [B, K, d] -> hd_pad [B, NP, d] (rows >= K zero) and dinv [B, NP]; one CTA per padded row
+constexpr int kPrepThreads = 256;
+__global__ void __launch_bounds__(kPrepThreads)
 draft_prep_kernel(const uint16_t *hd, int B, int K, int NP, int dim, uint16_t *hd_pad, float *dinv)
 {
-    const int r = blockIdx.x * kNormWarps + (threadIdx.x >> 5);   // padded row index over B * NP
-    const int lane = threadIdx.x & 31;
-    if (r >= B * NP) return;
+    __shared__ float part[kPrepThreads / 32];
+    const int r = blockIdx.x;                       // padded row index over B * NP
     const int b = r / NP, k = r - b * NP;
     uint4 *dst = reinterpret_cast<uint4 *>(hd_pad + (size_t)r * dim);
     if (k >= K) {
-        for (int i = lane; i < dim / 8; i += 32) dst[i] = make_uint4(0, 0, 0, 0);
-        if (lane == 0) dinv[r] = 0.f;
+        for (int i = threadIdx.x; i < dim / 8; i += kPrepThreads) dst[i] = make_uint4(0, 0, 0, 0);
+        if (threadIdx.x == 0) dinv[r] = 0.f;
         return;
     }
     const uint4 *src = reinterpret_cast<const uint4 *>(hd + ((size_t)b * K + k) * dim);
     float acc = 0.f;
-    for (int i = lane; i < dim / 8; i += 32) {
+    for (int i = threadIdx.x; i < dim / 8; i += kPrepThreads) {
         const uint4 w = __ldg(src + i);
         dst[i] = w;
         acc = sumsq_bf16x8(w, acc);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) dinv[r] = acc > 0.f ? 1.f / sqrtf(acc) : 0.f;
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int w = 0; w < kPrepThreads / 32; ++w) t += part[w];
+        dinv[r] = t > 0.f ? 1.f / sqrtf(t) : 0.f;
+    }
 }
 
 // ------------------------------------------------------------- cosine kernel
@@ -96,6 +102,7 @@ struct CosParams {
     int NP;                 // K padded to a multiple of 16 (MMA N)
     int smem_bytes;         // dynamic shared memory of the launch (after 1024-byte alignment)
     int tmem_cols;
+    int tail_a, tail_b;     // row-group counts that have a one-box tensor map of their own (0 = none)
     int n_grp;              // groups of 16 rows per batch element
     int total_groups;       // B * n_grp
 };
@@ -127,7 +134,8 @@ __device__ __forceinline__ bool wait_teardown(uint32_t bar, uint32_t parity)
 
 __global__ void __launch_bounds__(kCosThreads, 1)
 cos_tc_kernel(const CosParams P, const __grid_constant__ CUtensorMap tmap_v,
-              const __grid_constant__ CUtensorMap tmap_v128, const __grid_constant__ CUtensorMap tmap_d)
+              const __grid_constant__ CUtensorMap tmap_v128, const __grid_constant__ CUtensorMap tmap_va,
+              const __grid_constant__ CUtensorMap tmap_vb, const __grid_constant__ CUtensorMap tmap_d)
 {
     extern __shared__ uint8_t smem_raw[];
     const RelevanceParams &p = P.r;
@@ -174,6 +182,8 @@ cos_tc_kernel(const CosParams P, const __grid_constant__ CUtensorMap tmap_v,
         if (lane == 0) prefetch_tensormap(&tmap_v);
         if (lane == 1) prefetch_tensormap(&tmap_d);
         if (lane == 2) prefetch_tensormap(&tmap_v128);
+        if (lane == 3) prefetch_tensormap(&tmap_va);
+        if (lane == 4) prefetch_tensormap(&tmap_vb);
         const int n_bars = 2 * S + 6;
         for (int j = lane; j < n_bars; j += 32) {
             uint32_t count = 1;
@@ -218,9 +228,21 @@ cos_tc_kernel(const CosParams P, const __grid_constant__ CUtensorMap tmap_v,
                                          walk.b, stream_policy);
                         g = 16;
                     }
-                    for (; g < walk.n_groups; ++g)
-                        tma_load_3d_hint(dst + g * kGroupBytes, &tmap_v, full(s), kc * 64,
+                    // what is left of the chunk: in one box when its height is one of the
+                    // two the launch made maps for (issuing a TMA costs the producer
+                    // more than a hundred cycles), else in boxes of 16 rows
+                    const int left = walk.n_groups - g;
+                    if (left > 0 && left == P.tail_a) {
+                        tma_load_3d_hint(dst + g * kGroupBytes, &tmap_va, full(s), kc * 64,
                                          walk.row0 + g * 16, walk.b, stream_policy);
+                    } else if (left > 0 && left == P.tail_b) {
+                        tma_load_3d_hint(dst + g * kGroupBytes, &tmap_vb, full(s), kc * 64,
+                                         walk.row0 + g * 16, walk.b, stream_policy);
+                    } else {
+                        for (; g < walk.n_groups; ++g)
+                            tma_load_3d_hint(dst + g * kGroupBytes, &tmap_v, full(s), kc * 64,
+                                             walk.row0 + g * 16, walk.b, stream_policy);
+                    }
                     tma_load_3d(dst + d_off, &tmap_d, full(s), kc * 64, 0, walk.b);
                 }
             }
@@ -388,10 +410,38 @@ __global__ void __launch_bounds__(kTopThreads) topn_mean_kernel(const RelevanceP
             mine[i] = j < lv ? float_key(__ldcg(row + j)) : 0u;
             best = max(best, mine[i]);
         }
-        keys[tid] = best;
         if (tid == 0) n_cand = 0;
-        bitonic_sort_desc(keys, kTopThreads, tid);
-        const uint32_t bound = keys[n - 1];                 // >= n elements are at or above it
+        uint32_t bound;
+        if (n <= 32u) {
+            // the n-th largest of the 32 warp maxima: a looser bound, but one warp sorts
+            // 32 keys with shuffles alone
+            uint32_t wbest = best;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) wbest = max(wbest, __shfl_xor_sync(0xffffffffu, wbest, o));
+            if ((tid & 31) == 0) keys[tid >> 5] = wbest;
+            __syncthreads();
+            if (tid < 32) {
+                uint32_t x = keys[tid];
+#pragma unroll
+                for (int size = 2; size <= 32; size <<= 1) {
+#pragma unroll
+                    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+                        const uint32_t y = __shfl_xor_sync(0xffffffffu, x, stride);
+                        const bool upper = (tid & stride) != 0;          // holds the second of the pair
+                        const bool descending = (tid & size) == 0;
+                        const bool take_max = (upper != descending);     // first of a descending pair keeps the max
+                        x = take_max ? max(x, y) : min(x, y);
+                    }
+                }
+                keys[tid] = x;                                           // descending
+            }
+            __syncthreads();
+            bound = keys[n - 1];
+        } else {
+            keys[tid] = best;
+            bitonic_sort_desc(keys, kTopThreads, tid);
+            bound = keys[n - 1];                            // >= n elements are at or above it
+        }
         __syncthreads();
 #pragma unroll
         for (int i = 0; i < kTopPerThread; ++i) {
@@ -528,7 +578,7 @@ cudaError_t launch_visual_relevance(const RelevanceParams &p, cudaStream_t strea
     o = (o + 1023) & ~size_t(1023);
     float *dinv = reinterpret_cast<float *>(reinterpret_cast<char *>(p.cos_t) + o);
 
-    draft_prep_kernel<<<(p.B * NP + kNormWarps - 1) / kNormWarps, 32 * kNormWarps, 0, stream>>>(
+    draft_prep_kernel<<<p.B * NP, kPrepThreads, 0, stream>>>(
         p.h_draft, p.B, p.K, NP, p.d, hd_pad, dinv);
     ++*launches;
     cudaError_t err = cudaGetLastError();
@@ -544,10 +594,23 @@ cudaError_t launch_visual_relevance(const RelevanceParams &p, cudaStream_t strea
     P.tmem_cols = cols;
     P.n_grp = (p.lv + 15) / 16;
     P.total_groups = p.B * P.n_grp;
-    CUtensorMap mv, mv128, md;
+    // The shares are `per` or `per + 1` groups; what a share leaves after its full chunks
+    // and its full row block is the tail that gets a map of its own.
+    const int n_cta = P.total_groups < p.n_sm ? P.total_groups : p.n_sm;
+    auto tail_of = [](int groups) {
+        const int t = groups % kChunkGroups;
+        return t > 8 ? t - 8 : t;       // 0..8 groups
+    };
+    P.tail_a = tail_of(P.total_groups / n_cta);
+    P.tail_b = tail_of(P.total_groups / n_cta + 1);
+    if (P.tail_a * 16 > p.lv) P.tail_a = 0;
+    if (P.tail_b * 16 > p.lv) P.tail_b = 0;
+    CUtensorMap mv, mv128, mva, mvb, md;
     if (!make_rows_map(&mv, p.h_visual, p.d, p.lv, p.B, 16) ||
         // (fewer than 128 rows never make a full row block: the wide map is then not used)
         !make_rows_map(&mv128, p.h_visual, p.d, p.lv, p.B, p.lv >= 128 ? 128 : 16) ||
+        !make_rows_map(&mva, p.h_visual, p.d, p.lv, p.B, P.tail_a > 0 ? P.tail_a * 16 : 16) ||
+        !make_rows_map(&mvb, p.h_visual, p.d, p.lv, p.B, P.tail_b > 0 ? P.tail_b * 16 : 16) ||
         !make_rows_map(&md, hd_pad, p.d, NP, p.B, NP))
         return cudaErrorInvalidValue;
     const size_t smem = (size_t)P.smem_bytes + 1024;
@@ -557,13 +620,13 @@ cudaError_t launch_visual_relevance(const RelevanceParams &p, cudaStream_t strea
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(P.total_groups < p.n_sm ? P.total_groups : p.n_sm), 1, 1);
+    cfg.gridDim = dim3((unsigned)n_cta, 1, 1);
     cfg.blockDim = dim3(kCosThreads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    err = cudaLaunchKernelEx(&cfg, cos_tc_kernel, P, mv, mv128, md);
+    err = cudaLaunchKernelEx(&cfg, cos_tc_kernel, P, mv, mv128, mva, mvb, md);
     ++*launches;
     if (err != cudaSuccess) return err;
 
