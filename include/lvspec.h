@@ -123,6 +123,15 @@ uint64_t lvspec_launch_count(const lvspec_ctx_t *ctx);
 int32_t lvspec_attention_splits(const lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
                                 int32_t max_kv_len);
 
+/* Self-test of the bounded device-side waits.  Every barrier wait in the kernels
+ * of this library has a time limit (about two seconds); a wait that runs out
+ * raises LVSPEC_DEV_WAIT_EXPIRED and lets the kernel return, so that a lost
+ * arrival cannot hang the GPU.  This call enqueues one warp that waits, through
+ * the same code but with a limit of `limit_ms` milliseconds (1..2000), on a
+ * barrier nothing ever completes.  Afterwards lvspec_device_status reports
+ * LVSPEC_ERR_TIMEOUT once, and the context is as usable as before. */
+lvspec_status_t lvspec_selftest_wait_expiry(lvspec_ctx_t *ctx, int32_t limit_ms);
+
 /* ---- verification attention ---------------------------------------------------
  *
  * Operation (Eq. 1: the K draft tokens are verified by the target model in one

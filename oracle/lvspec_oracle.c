@@ -254,3 +254,38 @@ void lvspec_oracle_visual_relevance(const uint16_t *h_draft, const uint16_t *h_v
     }
 }
 
+/*
+ * What a verify step hands back to the decoding loop.  The paper defines the
+ * accepted length (Eq. 2) and is silent on the rest; this is the standard
+ * speculative-decoding bookkeeping under the rule's decisions:
+ *   - the first tau draft tokens are kept as they are (also at loosened or
+ *     shift-tolerated positions: the later target rows were computed with
+ *     exactly these tokens in the context);
+ *   - if a position was rejected (tau < gamma) the target's own token at that
+ *     position, y_tau, follows as the correction; with tau = gamma there is no
+ *     further target row to take a bonus token from;
+ *   - the cache keeps the accepted draft slots: new_kv_len = kv_len - gamma + tau
+ *     (the correction token has no K/V yet; it is the next step's input).
+ *
+ *   draft, target   int32 [B, gamma]
+ *   accept_len      int32 [B]
+ *   kv_len          int32 [B] or NULL
+ *   emitted         int32 [B, gamma]   tokens, -1 beyond n_emitted
+ *   n_emitted       int32 [B]          min(tau + 1, gamma)
+ *   new_kv_len      int32 [B]          (only with kv_len)
+ */
+void lvspec_oracle_emit(const int32_t *draft, const int32_t *target, const int32_t *accept_len,
+                        const int32_t *kv_len, int B, int gamma, int32_t *emitted,
+                        int32_t *n_emitted, int32_t *new_kv_len)
+{
+    for (int b = 0; b < B; ++b) {
+        const int tau = accept_len[b];
+        int n = 0;
+        for (int i = 0; i < gamma; ++i) emitted[(size_t)b * gamma + i] = -1;
+        for (int i = 0; i < tau; ++i) emitted[(size_t)b * gamma + n++] = draft[(size_t)b * gamma + i];
+        if (tau < gamma) emitted[(size_t)b * gamma + n++] = target[(size_t)b * gamma + tau];
+        n_emitted[b] = n;
+        if (kv_len && new_kv_len) new_kv_len[b] = kv_len[b] - gamma + tau;
+    }
+}
+

@@ -45,6 +45,8 @@ def _load():
         lib.lvspec_oracle_loose_accept.restype = None
         lib.lvspec_oracle_visual_relevance.argtypes = [p, p, i, i, i, i, i, p, p]
         lib.lvspec_oracle_visual_relevance.restype = None
+        lib.lvspec_oracle_emit.argtypes = [p, p, p, p, i, i, p, p, p]
+        lib.lvspec_oracle_emit.restype = None
         lib.lvspec_oracle_n_loose.argtypes = [ctypes.c_double, i]
         lib.lvspec_oracle_n_loose.restype = i
         try:
@@ -133,3 +135,20 @@ def visual_relevance(h_draft, h_visual, top_n: int, return_cosines: bool = False
     lib.lvspec_oracle_visual_relevance(_ptr(h_draft), _ptr(h_visual), B, K, lv, d, int(top_n),
                                        _ptr(rel), _ptr(cos))
     return (rel, cos) if return_cosines else rel
+
+
+def emit(draft, target, accept_len, kv_len=None):
+    """Tokens a verify step hands back: (emitted int32 [B,gamma] with -1 padding,
+    n_emitted int32 [B], new_kv_len int32 [B] or None)."""
+    lib = _load()
+    draft = np.ascontiguousarray(draft, dtype=np.int32)
+    target = np.ascontiguousarray(target, dtype=np.int32)
+    accept_len = np.ascontiguousarray(accept_len, dtype=np.int32)
+    B, gamma = draft.shape
+    emitted = np.empty((B, gamma), dtype=np.int32)
+    n_emitted = np.empty((B,), dtype=np.int32)
+    kv = None if kv_len is None else np.ascontiguousarray(kv_len, dtype=np.int32)
+    new_kv = None if kv is None else np.empty((B,), dtype=np.int32)
+    lib.lvspec_oracle_emit(_ptr(draft), _ptr(target), _ptr(accept_len), _ptr(kv), B, gamma,
+                           _ptr(emitted), _ptr(n_emitted), _ptr(new_kv))
+    return emitted, n_emitted, new_kv

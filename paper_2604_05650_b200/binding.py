@@ -29,6 +29,7 @@ EXPORTS = (
     "lvspec_attention_splits", "lvspec_verify_attention", "lvspec_verify_attention_host",
     "lvspec_loose_accept", "lvspec_loose_accept_ex", "lvspec_loose_accept_host",
     "lvspec_loose_accept_static", "lvspec_row_inv_norms", "lvspec_visual_relevance",
+    "lvspec_selftest_wait_expiry",
 )
 
 
@@ -82,6 +83,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lvspec_loose_accept.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp]
     lib.lvspec_loose_accept_ex.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp, vp, vp]
     lib.lvspec_loose_accept_host.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp]
+    lib.lvspec_selftest_wait_expiry.argtypes = [vp, i32]
     lib.lvspec_row_inv_norms.argtypes = [vp, ctypes.c_int64, i32, vp, vp]
     lib.lvspec_visual_relevance.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, i32, vp]
     lib.lvspec_loose_accept_static.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp,
@@ -146,6 +148,16 @@ class Context:
         if st not in (OK, ERR_TIMEOUT):
             self._check(st)
         return int(flags.value)
+
+    def device_status_code(self):
+        """(status code, flags) of ``lvspec_device_status``: the code is ERR_TIMEOUT
+        when a bounded device-side wait ran out since the last call."""
+        flags = ctypes.c_uint32(0)
+        st = self._lib.lvspec_device_status(self._h, ctypes.byref(flags))
+        return int(st), int(flags.value)
+
+    def selftest_wait_expiry(self, limit_ms: int = 5) -> None:
+        self._check(self._lib.lvspec_selftest_wait_expiry(self._h, int(limit_ms)))
 
     def launch_count(self) -> int:
         return int(self._lib.lvspec_launch_count(self._h))

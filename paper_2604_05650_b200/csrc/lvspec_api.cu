@@ -449,6 +449,19 @@ lvspec_status_t lvspec_verify_attention_host(lvspec_ctx_t *ctx, const lvspec_att
     return LVSPEC_OK;
 }
 
+lvspec_status_t lvspec_selftest_wait_expiry(lvspec_ctx_t *ctx, int32_t limit_ms)
+{
+    if (!ctx) return LVSPEC_ERR_INVALID_ARG;
+    if (limit_ms < 1 || limit_ms > 2000) return fail(ctx, LVSPEC_ERR_INVALID_ARG, "limit_ms outside 1..2000");
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
+    int launches = 0;
+    e = launch_wait_expiry(ctx->status, (unsigned long long)limit_ms * 1000000ull, ctx->stream, &launches);
+    ctx->launches += launches;
+    if (e != cudaSuccess) return cuda_fail(ctx, "self-test kernel launch", e);
+    return LVSPEC_OK;
+}
+
 lvspec_status_t lvspec_row_inv_norms(lvspec_ctx_t *ctx, int64_t rows, int32_t dim, const void *x,
                                      float *inv_norm)
 {

@@ -76,5 +76,7 @@ cudaError_t launch_row_inv_norms(const uint16_t *x, long long rows, int dim, flo
                                  cudaStream_t stream, int *launches);
 cudaError_t launch_visual_relevance(const RelevanceParams &p, cudaStream_t stream, int *launches);
 size_t relevance_scratch_bytes(int B, int K, int lv, int d);
+cudaError_t launch_wait_expiry(uint32_t *status, unsigned long long limit_ns, cudaStream_t stream,
+                               int *launches);
 
 }  // namespace lvspec

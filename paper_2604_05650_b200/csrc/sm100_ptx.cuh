@@ -65,24 +65,30 @@ __device__ __forceinline__ uint64_t global_timer_ns()
 }
 
 // Bounded wait: polls the barrier until the phase with the given parity has
-// completed, the CTA-wide abort flag is raised, or about two seconds pass.
-// Returns false when it gave up (and raises the abort flag itself).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+// completed, the CTA-wide abort flag is raised, or `limit_ns` pass.  Returns
+// false when it gave up (and raises the abort flag itself).
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                                uint64_t limit_ns)
 {
     if (mbar_try_wait(bar, parity)) return true;
     uint64_t t0 = 0;
     for (uint32_t spin = 1;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if ((spin & 1023u) == 0) {
+        if ((spin & 1023u) == 0 || limit_ns < 1000000ull) {
             const uint64_t now = global_timer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > 2000000000ull) {
+            else if (now - t0 > limit_ns) {
                 *abort_flag = 1;
                 return false;
             }
         }
     }
+}
+// The limit every kernel of this library uses: about two seconds.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    return mbar_wait_limit(bar, parity, abort_flag, 2000000000ull);
 }
 
 // ---- proxy / tcgen05 fences ---------------------------------------------------
