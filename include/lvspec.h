@@ -225,6 +225,30 @@ lvspec_status_t lvspec_loose_accept_ex(lvspec_ctx_t *ctx, int32_t batch, int32_t
                                        int32_t shift_window, int32_t *accept_len,
                                        int32_t *target_tokens, uint8_t *accepted);
 
+/* As lvspec_loose_accept, plus the emit step: what the verify step hands back
+ * to the decoding loop.  The paper defines the accepted length tau (Eq. 2) and
+ * is silent on the rest; this is the usual speculative-decoding bookkeeping
+ * under the rule's decisions.  The first tau draft tokens are kept as they are
+ * (also where they were accepted by loosening or by shift tolerance: the later
+ * target rows were computed with these very tokens in the context).  If a
+ * position was rejected (tau < gamma), the target's own token y_tau of that
+ * position follows as the correction; with tau = gamma there is no further
+ * target row to take a bonus token from.
+ *   kv_len      device, int32 [B]          optional (NULL together with new_kv_len)
+ *   emitted     device, int32 [B, gamma]   (written) tokens, -1 beyond n_emitted
+ *   n_emitted   device, int32 [B]          (written) min(tau + 1, gamma)
+ *   new_kv_len  device, int32 [B]          (written) kv_len - gamma + tau: the cache
+ *               keeps the accepted draft slots; the correction token has no K/V
+ *               yet and is the next step's input */
+lvspec_status_t lvspec_loose_accept_emit(lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,
+                                         int32_t vocab, int32_t n_mass_heads,
+                                         const float *target_logits, const int32_t *draft_tokens,
+                                         const float *visual_mass,
+                                         const lvspec_thresholds_t *thresholds,
+                                         int32_t shift_window, const int32_t *kv_len,
+                                         int32_t *accept_len, int32_t *emitted, int32_t *n_emitted,
+                                         int32_t *new_kv_len);
+
 /* Same operation on HOST buffers (see lvspec_verify_attention_host). */
 lvspec_status_t lvspec_loose_accept_host(lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,
                                          int32_t vocab, int32_t n_mass_heads,

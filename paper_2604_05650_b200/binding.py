@@ -29,7 +29,7 @@ EXPORTS = (
     "lvspec_attention_splits", "lvspec_verify_attention", "lvspec_verify_attention_host",
     "lvspec_loose_accept", "lvspec_loose_accept_ex", "lvspec_loose_accept_host",
     "lvspec_loose_accept_static", "lvspec_row_inv_norms", "lvspec_visual_relevance",
-    "lvspec_selftest_wait_expiry",
+    "lvspec_selftest_wait_expiry", "lvspec_loose_accept_emit",
 )
 
 
@@ -84,6 +84,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lvspec_loose_accept_ex.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp, vp, vp]
     lib.lvspec_loose_accept_host.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp]
     lib.lvspec_selftest_wait_expiry.argtypes = [vp, i32]
+    lib.lvspec_loose_accept_emit.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp, vp, vp, vp, vp]
     lib.lvspec_row_inv_norms.argtypes = [vp, ctypes.c_int64, i32, vp, vp]
     lib.lvspec_visual_relevance.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, i32, vp]
     lib.lvspec_loose_accept_static.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp,
@@ -203,6 +204,15 @@ class Context:
         self._check(self._lib.lvspec_visual_relevance(
             self._h, batch, gamma, n_visual, dim, _addr(h_draft), _addr(h_visual),
             _addr(visual_inv_norm), int(top_n), _addr(relevance)))
+
+    def loose_accept_emit(self, batch, gamma, vocab, n_mass_heads, target_logits, draft_tokens,
+                          visual_mass, accept_len, emitted, n_emitted, shift_window, lam: float = 0.7,
+                          n_loose: int = -1, kv_len=None, new_kv_len=None) -> None:
+        th = Thresholds(float(lam), int(n_loose), 0)
+        self._check(self._lib.lvspec_loose_accept_emit(
+            self._h, batch, gamma, vocab, n_mass_heads, _addr(target_logits), _addr(draft_tokens),
+            _addr(visual_mass), ctypes.byref(th), int(shift_window), _addr(kv_len), _addr(accept_len),
+            _addr(emitted), _addr(n_emitted), _addr(new_kv_len)))
 
     def loose_accept_host(self, batch, gamma, vocab, n_mass_heads, target_logits, draft_tokens,
                           visual_mass, accept_len, shift_window, lam: float = 0.7,

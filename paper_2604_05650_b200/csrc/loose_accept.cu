@@ -143,11 +143,27 @@ __global__ void __launch_bounds__(kThreads) loose_accept_kernel(const AcceptPara
         if (p.accepted) p.accepted[rid] = ok ? 1 : 0;
     }
     __syncthreads();
+    __shared__ int tau_s;
     if (tid == 0) {
         int tau = 0;
         while (tau < gamma && acc_s[tau]) ++tau;
         p.accept_len[b] = tau;
+        tau_s = tau;
         p.counters[b] = 0;                         // ready for the next call
+        // emit step: how many tokens go back to the decoding loop and how long the
+        // cache is afterwards (the accepted draft slots stay, the rest is dropped)
+        if (p.n_emitted) p.n_emitted[b] = min(tau + 1, gamma);
+        if (p.new_kv_len && p.kv_len) p.new_kv_len[b] = p.kv_len[b] - gamma + tau;
+    }
+    if (p.emitted) {
+        __syncthreads();
+        // accepted draft tokens as they are, then the target's own token at the
+        // rejected position, then -1
+        if (tid < gamma) {
+            const int tau = tau_s;
+            const int tok = tid < tau ? draft_s[tid] : (tid == tau ? y_s[tid] : -1);
+            p.emitted[(size_t)b * gamma + tid] = tok;
+        }
     }
 }
 

@@ -235,7 +235,8 @@ lvspec_status_t check_accept(lvspec_ctx *ctx, int batch, int gamma, int vocab, i
 lvspec_status_t run_accept(lvspec_ctx *ctx, int batch, int gamma, int vocab, int heads,
                            const float *logits, const int32_t *draft, const float *mass,
                            int n_loose, int window, int32_t *accept_len, int32_t *target,
-                           uint8_t *accepted)
+                           uint8_t *accepted, const int32_t *kv_len = nullptr, int32_t *emitted = nullptr,
+                           int32_t *n_emitted = nullptr, int32_t *new_kv_len = nullptr)
 {
     AcceptParams p;
     std::memset(&p, 0, sizeof p);
@@ -245,6 +246,10 @@ lvspec_status_t run_accept(lvspec_ctx *ctx, int batch, int gamma, int vocab, int
     p.accept_len = accept_len;
     p.target = target;
     p.accepted = accepted;
+    p.kv_len = kv_len;
+    p.emitted = emitted;
+    p.n_emitted = n_emitted;
+    p.new_kv_len = new_kv_len;
     p.counters = ctx->counters;
     p.status = ctx->status;
     p.B = batch;
@@ -547,6 +552,33 @@ lvspec_status_t lvspec_loose_accept_ex(lvspec_ctx_t *ctx, int32_t batch, int32_t
     if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
     return run_accept(ctx, batch, gamma, vocab, n_mass_heads, target_logits, draft_tokens,
                       visual_mass, n_loose, shift_window, accept_len, target_tokens, accepted);
+}
+
+lvspec_status_t lvspec_loose_accept_emit(lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,
+                                         int32_t vocab, int32_t n_mass_heads,
+                                         const float *target_logits, const int32_t *draft_tokens,
+                                         const float *visual_mass,
+                                         const lvspec_thresholds_t *thresholds,
+                                         int32_t shift_window, const int32_t *kv_len,
+                                         int32_t *accept_len, int32_t *emitted, int32_t *n_emitted,
+                                         int32_t *new_kv_len)
+{
+    int n_loose = 0;
+    lvspec_status_t st = check_accept(ctx, batch, gamma, vocab, n_mass_heads, target_logits,
+                                      draft_tokens, visual_mass, thresholds, shift_window,
+                                      accept_len, true, &n_loose);
+    if (st != LVSPEC_OK) return st;
+    if (!emitted || !n_emitted) return fail(ctx, LVSPEC_ERR_INVALID_ARG, "null argument");
+    if ((kv_len == nullptr) != (new_kv_len == nullptr))
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "kv_len and new_kv_len go together");
+    if ((reinterpret_cast<uintptr_t>(emitted) & 3u) || (reinterpret_cast<uintptr_t>(n_emitted) & 3u) ||
+        (reinterpret_cast<uintptr_t>(kv_len) & 3u) || (reinterpret_cast<uintptr_t>(new_kv_len) & 3u))
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "misaligned device pointer");
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
+    return run_accept(ctx, batch, gamma, vocab, n_mass_heads, target_logits, draft_tokens,
+                      visual_mass, n_loose, shift_window, accept_len, nullptr, nullptr, kv_len, emitted,
+                      n_emitted, new_kv_len);
 }
 
 lvspec_status_t lvspec_loose_accept(lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,

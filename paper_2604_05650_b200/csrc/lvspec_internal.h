@@ -53,6 +53,10 @@ struct AcceptParams {
     int32_t *accept_len;      // [B]
     int32_t *target;          // optional [B, gamma]
     uint8_t *accepted;        // optional [B, gamma]
+    const int32_t *kv_len;    // optional [B]: cache lengths going in (emit step)
+    int32_t *emitted;         // optional [B, gamma]: accepted draft tokens, then the correction token, then -1
+    int32_t *n_emitted;       // optional [B]
+    int32_t *new_kv_len;      // optional [B] (with kv_len)
     float *part_val;          // [B, gamma, n_vsplit]
     int32_t *part_idx;        // [B, gamma, n_vsplit]
     uint32_t *counters;       // [B], zero between calls

@@ -171,3 +171,43 @@ def test_invalid_arguments_launch_nothing(ctx):
     with pytest.raises(binding.LvspecError):
         ctx.loose_accept(1, 4, 100, 2, None, dr, ms, al, 1)
     assert ctx.launch_count() == before
+
+
+@pytest.mark.parametrize("cfg_id", [0, 2, 3])
+def test_emit_step(ctx, oracle_mod, cfg_id):
+    """Accepted draft tokens, correction token, token count and new cache length,
+    bit-exact against the oracle's emit step on the same inputs."""
+    import torch
+    cfg = W.CONFIGS[cfg_id]
+    B = 5
+    logits, draft = W.accept_inputs(cfg, batch=B)
+    mass = W.synthetic_mass(cfg, batch=B)
+    kv_len = np.array([cfg.kv_len - 3 * b for b in range(B)], dtype=np.int32)
+    n = oracle_mod.n_loose(cfg.lam, cfg.gamma)
+    for window in (0, cfg.shift_window):
+        tau, tgt, _ = oracle_mod.loose_accept(logits, draft, mass, n, window)
+        ref_em, ref_n, ref_kv = oracle_mod.emit(draft, tgt, tau, kv_len)
+        dl, dd, dm = (torch.from_numpy(x).cuda() for x in (logits, draft, mass))
+        dkv = torch.from_numpy(kv_len).cuda()
+        alen = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+        em = torch.full((B, cfg.gamma), -7, dtype=torch.int32, device="cuda")
+        ne = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+        nkv = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+        ctx.set_stream(torch.cuda.current_stream().cuda_stream)
+        ctx.loose_accept_emit(B, cfg.gamma, cfg.vocab, mass.shape[2], dl, dd, dm, alen, em, ne, window,
+                              n_loose=n, kv_len=dkv, new_kv_len=nkv)
+        torch.cuda.synchronize()
+        assert (alen.cpu().numpy() == tau).all()
+        assert (em.cpu().numpy() == ref_em).all()
+        assert (ne.cpu().numpy() == ref_n).all()
+        assert (nkv.cpu().numpy() == ref_kv).all()
+    # without cache lengths
+    ctx.loose_accept_emit(B, cfg.gamma, cfg.vocab, mass.shape[2], dl, dd, dm, alen, em, ne, window, n_loose=n)
+    torch.cuda.synchronize()
+    assert (em.cpu().numpy() == ref_em).all()
+    from paper_2604_05650_b200 import binding
+    with pytest.raises(binding.LvspecError):
+        ctx.loose_accept_emit(B, cfg.gamma, cfg.vocab, mass.shape[2], dl, dd, dm, alen, em, ne, window,
+                              n_loose=n, kv_len=dkv)          # kv_len without new_kv_len
+    with pytest.raises(binding.LvspecError):
+        ctx.loose_accept_emit(B, cfg.gamma, cfg.vocab, mass.shape[2], dl, dd, dm, alen, None, ne, window, n_loose=n)

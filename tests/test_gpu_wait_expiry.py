@@ -28,7 +28,7 @@ def test_expired_wait_is_reported_and_the_context_stays_usable(oracle_mod):
         assert 0.015 <= waited < 1.5, waited
         assert ctx.device_status_code() == (binding.OK, 0)   # reported once, then cleared
         # the context and the device still work
-        cfg = W.sweep_config(gamma=4, kv_len=1024, batch=1)
+        cfg = W.sweep_config(gamma=4, kv_len=2048, batch=1)
         case = W.attention_inputs(cfg)
         out, mass = run_attention(ctx, *case)
         ref_out, ref_mass = oracle_mod.verify_attention(*case)
