@@ -1,6 +1,6 @@
 """CPU oracle of the LVSpec verify step (test infrastructure, fp64, plain C)."""
 from .oracle import (build, verify_attention, loose_accept, n_loose, set_threads,
-                     max_threads, visual_relevance, emit)
+                     max_threads, visual_relevance, emit, select_branch)
 
 __all__ = ["build", "verify_attention", "loose_accept", "n_loose", "set_threads",
-           "max_threads", "visual_relevance", "emit"]
+           "max_threads", "visual_relevance", "emit", "select_branch"]

@@ -45,11 +45,32 @@ static double bf16_to_double(uint16_t bits)
  *
  * Query g of a sequence sees positions j < kv_len - gamma + g + 1 (causal over
  * the draft tail).  Head h reads KV head h / (Hq / Hkv).
+ *
+ * Draft-token trees (App. "Exploration on Draft Token Trees": a static tree of
+ * branches with K draft tokens each, every branch verified on its own): the
+ * gamma = R * branch_len draft slots at the end of the cache hold the branches
+ * one after the other, and query g (branch g / branch_len) sees the context
+ * before the draft slots plus the slots of its own branch up to itself.
+ * branch_len = gamma is the plain chain above.
  */
+void lvspec_oracle_verify_attention_tree(const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                                         const int32_t *kv_len, const int32_t *span,
+                                         int B, int gamma, int branch_len, int Hq, int Hkv, int D,
+                                         int Lmax, double *out, double *mass, double *probs);
+
 void lvspec_oracle_verify_attention(const uint16_t *q, const uint16_t *k, const uint16_t *v,
                                     const int32_t *kv_len, const int32_t *span,
                                     int B, int gamma, int Hq, int Hkv, int D, int Lmax,
                                     double *out, double *mass, double *probs)
+{
+    lvspec_oracle_verify_attention_tree(q, k, v, kv_len, span, B, gamma, gamma, Hq, Hkv, D, Lmax, out,
+                                        mass, probs);
+}
+
+void lvspec_oracle_verify_attention_tree(const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                                         const int32_t *kv_len, const int32_t *span,
+                                         int B, int gamma, int branch_len, int Hq, int Hkv, int D,
+                                         int Lmax, double *out, double *mass, double *probs)
 {
     const int G = Hq / Hkv;
     const double scale = 1.0 / sqrt((double)D);
@@ -64,7 +85,9 @@ void lvspec_oracle_verify_attention(const uint16_t *q, const uint16_t *k, const 
             const int g = (int)((u / Hq) % gamma);
             const int b = (int)(u / ((long)Hq * gamma));
             const int kvh = h / G;
-            const int vis = kv_len[b] - gamma + g + 1;
+            const int ctx_len = kv_len[b] - gamma;              /* positions before the draft slots */
+            const int own0 = ctx_len + (g / branch_len) * branch_len;   /* first slot of g's branch */
+            const int vis = kv_len[b] - gamma + g + 1;          /* one past g's own slot */
             const int vs = span[2 * b], ve = span[2 * b + 1];
             const uint16_t *qrow = q + (((size_t)b * gamma + g) * Hq + h) * D;
             const uint16_t *kb = k + ((size_t)b * Hkv + kvh) * (size_t)Lmax * D;
@@ -74,19 +97,21 @@ void lvspec_oracle_verify_attention(const uint16_t *q, const uint16_t *k, const 
             for (int d = 0; d < D; ++d) qd[d] = bf16_to_double(qrow[d]);
             double m = -INFINITY;
             for (int j = 0; j < vis; ++j) {
+                if (j >= ctx_len && j < own0) { s[j] = -INFINITY; continue; }   /* another branch */
                 double acc = 0.0;
                 for (int d = 0; d < D; ++d) acc += qd[d] * bf16_to_double(kb[(size_t)j * D + d]);
                 s[j] = acc * scale;
                 if (s[j] > m) m = s[j];
             }
             double Z = 0.0;
-            for (int j = 0; j < vis; ++j) { s[j] = exp(s[j] - m); Z += s[j]; }
+            for (int j = 0; j < vis; ++j) { s[j] = (s[j] == -INFINITY) ? 0.0 : exp(s[j] - m); Z += s[j]; }
             for (int d = 0; d < D; ++d) orow[d] = 0.0;
             double vm = 0.0;
             for (int j = 0; j < vis; ++j) {
                 const double p = s[j] / Z;
                 if (j >= vs && j < ve) vm += p;
-                for (int d = 0; d < D; ++d) orow[d] += p * bf16_to_double(vb[(size_t)j * D + d]);
+                if (p != 0.0)
+                    for (int d = 0; d < D; ++d) orow[d] += p * bf16_to_double(vb[(size_t)j * D + d]);
                 if (probs) probs[(((size_t)b * gamma + g) * Hq + h) * (size_t)Lmax + j] = p;
             }
             if (probs)
@@ -286,6 +311,24 @@ void lvspec_oracle_emit(const int32_t *draft, const int32_t *target, const int32
         if (tau < gamma) emitted[(size_t)b * gamma + n++] = target[(size_t)b * gamma + tau];
         n_emitted[b] = n;
         if (kv_len && new_kv_len) new_kv_len[b] = kv_len[b] - gamma + tau;
+    }
+}
+
+/*
+ * Draft-token trees: after every branch has been verified on its own (one
+ * accepted length per branch), the branch with the longest accepted length is
+ * kept; among equals the first.
+ *   accept_len  int32 [B, R]  ->  best_branch int32 [B], best_len int32 [B]
+ */
+void lvspec_oracle_select_branch(const int32_t *accept_len, int B, int R, int32_t *best_branch,
+                                 int32_t *best_len)
+{
+    for (int b = 0; b < B; ++b) {
+        int best = 0;
+        for (int r = 1; r < R; ++r)
+            if (accept_len[(size_t)b * R + r] > accept_len[(size_t)b * R + best]) best = r;
+        best_branch[b] = best;
+        best_len[b] = accept_len[(size_t)b * R + best];
     }
 }
 

@@ -41,6 +41,10 @@ def _load():
         i = ctypes.c_int
         lib.lvspec_oracle_verify_attention.argtypes = [p, p, p, p, p, i, i, i, i, i, i, p, p, p]
         lib.lvspec_oracle_verify_attention.restype = None
+        lib.lvspec_oracle_verify_attention_tree.argtypes = [p, p, p, p, p, i, i, i, i, i, i, i, p, p, p]
+        lib.lvspec_oracle_verify_attention_tree.restype = None
+        lib.lvspec_oracle_select_branch.argtypes = [p, i, i, p, p]
+        lib.lvspec_oracle_select_branch.restype = None
         lib.lvspec_oracle_loose_accept.argtypes = [p, p, p, i, i, i, i, i, i, p, p, p]
         lib.lvspec_oracle_loose_accept.restype = None
         lib.lvspec_oracle_visual_relevance.argtypes = [p, p, i, i, i, i, i, p, p]
@@ -75,9 +79,10 @@ def _ptr(a):
     return a.ctypes.data_as(ctypes.c_void_p) if a is not None else None
 
 
-def verify_attention(q, k, v, kv_len, span, return_probs: bool = False):
+def verify_attention(q, k, v, kv_len, span, return_probs: bool = False, branch_len: int = 0):
     """q [B,gamma,Hq,D], k/v [B,Hkv,Lmax,D] as uint16 bf16 bit patterns;
-    kv_len int32 [B]; span int32 [B,2].  Returns (out, mass[, probs]) in fp64."""
+    kv_len int32 [B]; span int32 [B,2].  Returns (out, mass[, probs]) in fp64.
+    ``branch_len`` > 0: the gamma draft slots are gamma / branch_len tree branches."""
     lib = _load()
     q = np.ascontiguousarray(q, dtype=np.uint16)
     k = np.ascontiguousarray(k, dtype=np.uint16)
@@ -92,9 +97,11 @@ def verify_attention(q, k, v, kv_len, span, return_probs: bool = False):
     out = np.empty((B, gamma, Hq, D), dtype=np.float64)
     mass = np.empty((B, gamma, Hq), dtype=np.float64)
     probs = np.empty((B, gamma, Hq, Lmax), dtype=np.float64) if return_probs else None
-    lib.lvspec_oracle_verify_attention(_ptr(q), _ptr(k), _ptr(v), _ptr(kv_len), _ptr(span),
-                                       B, gamma, Hq, Hkv, D, Lmax, _ptr(out), _ptr(mass),
-                                       _ptr(probs))
+    bl = gamma if branch_len <= 0 else int(branch_len)
+    assert gamma % bl == 0
+    lib.lvspec_oracle_verify_attention_tree(_ptr(q), _ptr(k), _ptr(v), _ptr(kv_len), _ptr(span),
+                                            B, gamma, bl, Hq, Hkv, D, Lmax, _ptr(out), _ptr(mass),
+                                            _ptr(probs))
     return (out, mass, probs) if return_probs else (out, mass)
 
 
@@ -152,3 +159,14 @@ def emit(draft, target, accept_len, kv_len=None):
     lib.lvspec_oracle_emit(_ptr(draft), _ptr(target), _ptr(accept_len), _ptr(kv), B, gamma,
                            _ptr(emitted), _ptr(n_emitted), _ptr(new_kv))
     return emitted, n_emitted, new_kv
+
+
+def select_branch(accept_len):
+    """accept_len int32 [B,R] -> (best_branch int32 [B], best_len int32 [B])."""
+    lib = _load()
+    a = np.ascontiguousarray(accept_len, dtype=np.int32)
+    B, R = a.shape
+    bb = np.empty((B,), dtype=np.int32)
+    bl = np.empty((B,), dtype=np.int32)
+    lib.lvspec_oracle_select_branch(_ptr(a), B, R, _ptr(bb), _ptr(bl))
+    return bb, bl
