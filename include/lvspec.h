@@ -167,6 +167,36 @@ lvspec_status_t lvspec_verify_attention(lvspec_ctx_t *ctx, const lvspec_attn_sha
                                         const int32_t *kv_len, const int32_t *visual_span,
                                         void *out, float *visual_mass);
 
+/* Draft-token trees (App. "Exploration on Draft Token Trees": a static tree of
+ * branches with K draft tokens each; every branch is verified loosely on its
+ * own and the branch with the longest accepted length is kept).
+ *
+ * lvspec_verify_attention_tree is lvspec_verify_attention for such a tree:
+ * shape->gamma counts ALL draft queries, gamma = n_branches * K; the gamma draft
+ * slots at the end of the cache hold the branches one after the other; query g
+ * (branch g / K) sees the context before the draft slots and the slots of its
+ * own branch up to itself, nothing of the other branches.  All else, limits
+ * included (gamma * Hq / Hkv <= LVSPEC_MAX_ROWS), is as for
+ * lvspec_verify_attention; n_branches = 1 is that call.
+ *
+ * The acceptance pass then treats the branches as sequences of their own:
+ * lvspec_loose_accept with batch = B * n_branches and gamma = K on logits
+ * [B, n_branches, K, V], drafts [B, n_branches, K] and the attention's
+ * visual_mass [B, n_branches * K, Hq] read as [B * n_branches, K, Hq]; the
+ * loosened set is taken among the K positions of a branch.
+ * lvspec_select_branch picks, per sequence, the branch with the longest accepted
+ * length (the first among equals):
+ *   accept_len   device, int32 [B, n_branches]
+ *   best_branch  device, int32 [B]   (written)
+ *   best_len     device, int32 [B]   (written)
+ * B * n_branches <= LVSPEC_MAX_BATCH. */
+lvspec_status_t lvspec_verify_attention_tree(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                             int32_t n_branches, const void *q, const void *k_cache,
+                                             const void *v_cache, const int32_t *kv_len,
+                                             const int32_t *visual_span, void *out, float *visual_mass);
+lvspec_status_t lvspec_select_branch(lvspec_ctx_t *ctx, int32_t batch, int32_t n_branches,
+                                     const int32_t *accept_len, int32_t *best_branch, int32_t *best_len);
+
 /* Same operation on HOST buffers: copies q, the caches, and the results through
  * device staging memory the context owns (grown on demand), on the context's
  * stream, and synchronises before returning.  All seven arrays are host

@@ -30,6 +30,7 @@ EXPORTS = (
     "lvspec_loose_accept", "lvspec_loose_accept_ex", "lvspec_loose_accept_host",
     "lvspec_loose_accept_static", "lvspec_row_inv_norms", "lvspec_visual_relevance",
     "lvspec_selftest_wait_expiry", "lvspec_loose_accept_emit",
+    "lvspec_verify_attention_tree", "lvspec_select_branch",
 )
 
 
@@ -84,6 +85,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lvspec_loose_accept_ex.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp, vp, vp]
     lib.lvspec_loose_accept_host.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp]
     lib.lvspec_selftest_wait_expiry.argtypes = [vp, i32]
+    lib.lvspec_verify_attention_tree.argtypes = [vp, S, i32, vp, vp, vp, vp, vp, vp, vp]
+    lib.lvspec_select_branch.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.lvspec_loose_accept_emit.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp, vp, vp, vp, vp]
     lib.lvspec_row_inv_norms.argtypes = [vp, ctypes.c_int64, i32, vp, vp]
     lib.lvspec_visual_relevance.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, i32, vp]
@@ -175,6 +178,19 @@ class Context:
         self._check(self._lib.lvspec_verify_attention(
             self._h, ctypes.byref(shape), _addr(q), _addr(k_cache), _addr(v_cache),
             kv_len.ctypes.data, span.ctypes.data, _addr(out), _addr(visual_mass)))
+
+    def verify_attention_tree(self, shape: AttnShape, n_branches, q, k_cache, v_cache, kv_len, visual_span,
+                              out, visual_mass) -> None:
+        kv_len, span = _i32(kv_len), _i32(visual_span)
+        if shape.batch >= 1 and (kv_len.size != shape.batch or span.size != 2 * shape.batch):
+            raise ValueError("kv_len needs B entries and visual_span B pairs")
+        self._check(self._lib.lvspec_verify_attention_tree(
+            self._h, ctypes.byref(shape), int(n_branches), _addr(q), _addr(k_cache), _addr(v_cache),
+            kv_len.ctypes.data, span.ctypes.data, _addr(out), _addr(visual_mass)))
+
+    def select_branch(self, batch, n_branches, accept_len, best_branch, best_len) -> None:
+        self._check(self._lib.lvspec_select_branch(self._h, int(batch), int(n_branches), _addr(accept_len),
+                                                   _addr(best_branch), _addr(best_len)))
 
     def verify_attention_host(self, shape: AttnShape, q, k_cache, v_cache, kv_len, visual_span,
                               out, visual_mass) -> None:

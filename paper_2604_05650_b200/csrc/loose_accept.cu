@@ -167,7 +167,31 @@ __global__ void __launch_bounds__(kThreads) loose_accept_kernel(const AcceptPara
     }
 }
 
+// Draft-token trees: one accepted length per branch goes in, the branch with the
+// longest one (the first among equals) comes out.  One thread per sequence.
+__global__ void select_branch_kernel(const int32_t *accept_len, int B, int R, int32_t *best_branch,
+                                     int32_t *best_len)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    int best = 0, len = accept_len[(size_t)b * R];
+    for (int r = 1; r < R; ++r) {
+        const int l = accept_len[(size_t)b * R + r];
+        if (l > len) { len = l; best = r; }
+    }
+    best_branch[b] = best;
+    best_len[b] = len;
+}
+
 }  // namespace
+
+cudaError_t launch_select_branch(const int32_t *accept_len, int B, int R, int32_t *best_branch,
+                                 int32_t *best_len, cudaStream_t stream, int *launches)
+{
+    select_branch_kernel<<<(B + 127) / 128, 128, 0, stream>>>(accept_len, B, R, best_branch, best_len);
+    ++*launches;
+    return cudaGetLastError();
+}
 
 cudaError_t launch_loose_accept(const AcceptParams &p, cudaStream_t stream, int *launches)
 {

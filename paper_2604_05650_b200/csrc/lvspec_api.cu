@@ -150,7 +150,7 @@ lvspec_status_t check_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, c
 
 lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, const SeqInfo &seq,
                               int max_len, const void *q, const void *k, const void *v, void *out,
-                              float *mass)
+                              float *mass, int branch_len = 0)
 {
     AttnParams p;
     std::memset(&p, 0, sizeof p);
@@ -171,6 +171,7 @@ lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, con
     p.n_split = s->n_split > 0 ? s->n_split : choose_splits(ctx, s, max_len);
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)p.D));
     p.pdl = ctx->pdl ? 1 : 0;
+    p.branch_len = branch_len > 0 ? branch_len : p.gamma;
 
     const size_t o_bytes = part_o_elems(p) * sizeof(float);
     const size_t st_bytes = part_stat_elems(p) * sizeof(float);
@@ -418,6 +419,24 @@ lvspec_status_t lvspec_verify_attention(lvspec_ctx_t *ctx, const lvspec_attn_sha
     return run_attention(ctx, shape, seq, max_len, q, k_cache, v_cache, out, visual_mass);
 }
 
+lvspec_status_t lvspec_verify_attention_tree(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                             int32_t n_branches, const void *q, const void *k_cache,
+                                             const void *v_cache, const int32_t *kv_len,
+                                             const int32_t *visual_span, void *out, float *visual_mass)
+{
+    SeqInfo seq;
+    int max_len = 0;
+    lvspec_status_t st = check_attention(ctx, shape, q, k_cache, v_cache, kv_len, visual_span, out,
+                                         visual_mass, true, &seq, &max_len);
+    if (st != LVSPEC_OK) return st;
+    if (n_branches < 1 || shape->gamma % n_branches != 0)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "gamma must be a positive multiple of n_branches");
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
+    return run_attention(ctx, shape, seq, max_len, q, k_cache, v_cache, out, visual_mass,
+                         shape->gamma / n_branches);
+}
+
 lvspec_status_t lvspec_verify_attention_host(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
                                              const void *q, const void *k_cache,
                                              const void *v_cache, const int32_t *kv_len,
@@ -451,6 +470,25 @@ lvspec_status_t lvspec_verify_attention_host(lvspec_ctx_t *ctx, const lvspec_att
         (e = cudaMemcpyAsync(visual_mass, dm, m_bytes, cudaMemcpyDeviceToHost, ctx->stream)) != cudaSuccess ||
         (e = cudaStreamSynchronize(ctx->stream)) != cudaSuccess)
         return cuda_fail(ctx, "device to host copy", e);
+    return LVSPEC_OK;
+}
+
+lvspec_status_t lvspec_select_branch(lvspec_ctx_t *ctx, int32_t batch, int32_t n_branches,
+                                     const int32_t *accept_len, int32_t *best_branch, int32_t *best_len)
+{
+    if (!ctx) return LVSPEC_ERR_INVALID_ARG;
+    if (!accept_len || !best_branch || !best_len) return fail(ctx, LVSPEC_ERR_INVALID_ARG, "null argument");
+    if (batch < 1 || n_branches < 1 || (long long)batch * n_branches > LVSPEC_MAX_BATCH)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "batch * n_branches outside 1..LVSPEC_MAX_BATCH");
+    if ((reinterpret_cast<uintptr_t>(accept_len) & 3u) || (reinterpret_cast<uintptr_t>(best_branch) & 3u) ||
+        (reinterpret_cast<uintptr_t>(best_len) & 3u))
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "misaligned device pointer");
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
+    int launches = 0;
+    e = launch_select_branch(accept_len, batch, n_branches, best_branch, best_len, ctx->stream, &launches);
+    ctx->launches += launches;
+    if (e != cudaSuccess) return cuda_fail(ctx, "branch selection kernel launch", e);
     return LVSPEC_OK;
 }
 

@@ -26,8 +26,18 @@ struct AttnParams {
     uint32_t *status;      // device status word
     int32_t B, gamma, Hq, Hkv, D, Lmax, G, M, n_split;
     int32_t pdl;           // launch programmatically dependent on the previous kernel
+    int32_t branch_len;    // draft tokens per tree branch (= gamma for a plain chain)
     float scale_log2;      // log2(e) / sqrt(D)
 };
+
+// Does draft query `qi` see the cache position with tail index t = pos - (kv_len -
+// gamma)?  t < 0 is the context before the draft slots: always visible.  Among
+// the draft slots a query sees its own branch up to itself (branches of
+// `branch_len` slots sit one after the other; a plain chain is one branch).
+__host__ __device__ inline bool draft_query_sees(int qi, int t, int branch_len)
+{
+    return qi >= t && (t < 0 || (qi / branch_len) * branch_len <= t);
+}
 
 // Partial results of one KV split, rows r = g * G + hg.
 static inline size_t part_o_elems(const AttnParams &p)
@@ -64,6 +74,8 @@ struct AcceptParams {
     int32_t B, gamma, V, Hm, n_loose, window, n_vsplit;
 };
 cudaError_t launch_loose_accept(const AcceptParams &p, cudaStream_t stream, int *launches);
+cudaError_t launch_select_branch(const int32_t *accept_len, int B, int R, int32_t *best_branch,
+                                 int32_t *best_len, cudaStream_t stream, int *launches);
 
 struct RelevanceParams {
     const uint16_t *h_draft;    // [B, K, d] bf16

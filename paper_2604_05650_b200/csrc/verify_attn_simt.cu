@@ -129,7 +129,7 @@ attn_simt_kernel(const AttnParams p, const SeqInfo seq)
         for (int r = warp; r < M; r += kThreads / 32) {
             const int g = r / G;
             const int pos = pos0 + lane;
-            const bool visible = pos < L - gamma + g + 1;
+            const bool visible = pos < L && draft_query_sees(g, pos - (L - gamma), p.branch_len);
             const float s = visible ? s_s[r * kTile + lane] : -INFINITY;
             float mx = s;
 #pragma unroll

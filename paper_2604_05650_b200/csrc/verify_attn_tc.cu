@@ -116,7 +116,7 @@ __device__ __forceinline__ bool group_any(int id, bool pred)
 
 // exp2 of eight scaled scores of one position, packed to bf16; returns their maximum
 __device__ __forceinline__ float exp_chunk(const uint32_t (&r)[8], const float *m8, float scale,
-                                           bool tail, int col0, int G, int gmin, uint4 &dst)
+                                           bool tail, int col0, int G, int gmin, int branch_len, uint4 &dst)
 {
     const float4 ma = *reinterpret_cast<const float4 *>(m8);
     const float4 mb = *reinterpret_cast<const float4 *>(m8 + 4);
@@ -126,7 +126,8 @@ __device__ __forceinline__ float exp_chunk(const uint32_t (&r)[8], const float *
     for (int k = 0; k < 8; ++k) x[k] = fmaf(__uint_as_float(r[k]), scale, -mm[k]);
     if (tail) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) x[k] = ((col0 + k) / G >= gmin) ? x[k] : -INFINITY;
+        for (int k = 0; k < 8; ++k)
+            x[k] = draft_query_sees((col0 + k) / G, gmin, branch_len) ? x[k] : -INFINITY;
     }
     float mx = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])),
                      fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
@@ -480,7 +481,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 group_sync(bar_id);
             }
             const bool tail = pos0 + kTilePos > L - gamma;
-            const int gmin = pos - L + gamma;           // queries g < gmin do not see `pos`
+            const int gmin = pos - L + gamma;           // tail index of `pos`: queries below it do not see it
             uint8_t *prow = gbase + sm.p + pb * (NP * 256) + row * 16;
             uint4 pk[kMaxChunks];   // this position's probabilities, 8 columns per entry
 
@@ -499,7 +500,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                         for (int u = 0; u < 4; ++u)
                             if (4 * h + u < kMaxChunks && cb + u < c_hi)
                                 gmax = fmaxf(gmax, exp_chunk(r[u], m_s + (cb + u) * 8, scale, tail,
-                                                             (cb + u) * 8, G, gmin, pk[4 * h + u]));
+                                                             (cb + u) * 8, G, gmin, p.branch_len, pk[4 * h + u]));
                     }
                 }
                 if (!group_any(bar_id, gmax > kGuard)) break;
@@ -512,7 +513,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
                         float s2 = __uint_as_float(r[k]) * scale;
-                        if (tail && (c8 * 8 + k) / G < gmin) s2 = -INFINITY;
+                        if (tail && !draft_query_sees((c8 * 8 + k) / G, gmin, p.branch_len)) s2 = -INFINITY;
 #pragma unroll
                         for (int o = 16; o > 0; o >>= 1)
                             s2 = fmaxf(s2, __shfl_xor_sync(0xffffffffu, s2, o));
