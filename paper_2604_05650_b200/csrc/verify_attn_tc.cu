@@ -61,7 +61,7 @@ struct TcConfig {
 
 // Byte offsets of the shared-memory regions (relative to a 1024-aligned base).
 struct SmemMap {
-    uint32_t k, v, q, p, a2, m, dl, tmx, bars, misc, total;
+    uint32_t k, v, q, p, a2, m, dl, tmx, vis, bars, misc, total;
 };
 __host__ __device__ inline SmemMap smem_map(const TcConfig &c)
 {
@@ -75,6 +75,7 @@ __host__ __device__ inline SmemMap smem_map(const TcConfig &c)
     s.m = o;    o += c.n_pad * 4;
     s.dl = o;   o += c.n_pad * 4;
     s.tmx = o;  o += 4 * c.n_pad * 4;
+    s.vis = o;  o += c.n_pad * 8;
     s.bars = o; o += 8 * (2 * c.ks + 2 * c.vs + 4 + 2 * c.pb + 3);
     s.misc = o; o += 16;
     s.total = o;
@@ -114,9 +115,19 @@ __device__ __forceinline__ bool group_any(int id, bool pred)
     return out != 0;
 }
 
+// Which draft slots a column's query sees: tail indices [lo, hi] (its own branch up to
+// itself); the context before the draft slots (tail index < 0) is visible to all.
+__device__ __forceinline__ bool column_sees(int2 lohi, int t)
+{
+    return t < 0 || (unsigned)(t - lohi.x) <= (unsigned)(lohi.y - lohi.x);
+}
+
 // exp2 of eight scaled scores of one position, packed to bf16; returns their maximum
+// kMask: 0 = every column sees the position; 1 = plain chain of draft tokens (query
+// col / G sees tail index t iff it is not below t); 2 = draft tree (table look-up)
+template <int kMask>
 __device__ __forceinline__ float exp_chunk(const uint32_t (&r)[8], const float *m8, float scale,
-                                           bool tail, int col0, int G, int gmin, int branch_len, uint4 &dst)
+                                           const int2 *vis8, int col0, int G, int t, uint4 &dst)
 {
     const float4 ma = *reinterpret_cast<const float4 *>(m8);
     const float4 mb = *reinterpret_cast<const float4 *>(m8 + 4);
@@ -124,10 +135,12 @@ __device__ __forceinline__ float exp_chunk(const uint32_t (&r)[8], const float *
     float x[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k) x[k] = fmaf(__uint_as_float(r[k]), scale, -mm[k]);
-    if (tail) {
+    if (kMask == 1) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
-            x[k] = draft_query_sees((col0 + k) / G, gmin, branch_len) ? x[k] : -INFINITY;
+        for (int k = 0; k < 8; ++k) x[k] = ((col0 + k) / G >= t) ? x[k] : -INFINITY;
+    } else if (kMask == 2) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) x[k] = column_sees(vis8[k], t) ? x[k] : -INFINITY;
     }
     float mx = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])),
                      fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
@@ -140,6 +153,38 @@ __device__ __forceinline__ float exp_chunk(const uint32_t (&r)[8], const float *
     return mx;
 }
 
+// One pass over this thread's position: exp2 of its chunks [c_lo, c_hi) of S^T (up to
+// four TMEM loads in flight per wait), packed probabilities into pk, returns the
+// largest scaled score.  kMask != 0: the tile reaches into the draft slots, so
+// columns are masked by what their query may see; the common tile carries none of that.
+template <int kMask>
+__device__ __forceinline__ float softmax_pass(uint32_t s_addr, int c_lo, int c_hi, const float *m_s,
+                                              float scale, const int2 *vis_s, int G, int t,
+                                              uint4 (&pk)[kMaxChunks])
+{
+    float gmax = -INFINITY;
+#pragma unroll
+    for (int h = 0; h < (kMaxChunks + 3) / 4; ++h) {
+        const int cb = c_lo + 4 * h;
+        if (cb < c_hi) {
+            uint32_t r[4][8];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (4 * h + u < kMaxChunks && cb + u < c_hi) tmem_ld_x8(s_addr + (cb + u) * 8, r[u]);
+            tmem_wait_ld();
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (4 * h + u < kMaxChunks && cb + u < c_hi)
+                    gmax = fmaxf(gmax, exp_chunk<kMask>(r[u], m_s + (cb + u) * 8, scale, vis_s + (cb + u) * 8,
+                                                        (cb + u) * 8, G, t, pk[4 * h + u]));
+        }
+    }
+    return gmax;
+}
+
+// kTree: the draft slots hold several branches (the visibility table is only built
+// and read then; the plain chain keeps its arithmetic mask)
+template <bool kTree>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUtensorMap tmap_k,
                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_q)
@@ -179,6 +224,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     float *m_s = reinterpret_cast<float *>(gbase + sm.m);
     float *dl_s = reinterpret_cast<float *>(gbase + sm.dl);
     float *tmx_s = reinterpret_cast<float *>(gbase + sm.tmx);
+    int2 *vis_s = reinterpret_cast<int2 *>(gbase + sm.vis);
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gbase + sm.misc);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(gbase + sm.misc + 4);
 
@@ -270,7 +316,15 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         // P buffers start as zeros (columns beyond the last chunk stay zero)
         for (uint32_t i = idx * 16; i < (uint32_t)(cfg.pb * NP * 256); i += kSoftmaxThreads * 16)
             *reinterpret_cast<uint4 *>(gbase + sm.p + i) = make_uint4(0, 0, 0, 0);
-        for (int n = idx; n < NP; n += kSoftmaxThreads) m_s[n] = 0.f;
+        for (int n = idx; n < NP; n += kSoftmaxThreads) {
+            m_s[n] = 0.f;
+            if (kTree) {
+                // the draft slots column n's query sees: its branch's first slot .. its own slot
+                const int qi = n / G;
+                vis_s[n] = qi < gamma ? make_int2((qi / p.branch_len) * p.branch_len, qi)
+                                      : make_int2(1 << 30, (1 << 30) - 1);
+            }
+        }
         // constant 64 x 16 tiles (K-major, no swizzle: the 8 positions of chunk c
         // at c * 1024, row r at (r / 8) * 128 + (r % 8) * 16).  Row 0 = ones (sums
         // l), row 1 = 1 inside the visual span (sums l_vis), rows 2.. = 0.
@@ -486,23 +540,9 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             uint4 pk[kMaxChunks];   // this position's probabilities, 8 columns per entry
 
             for (int attempt = 0; attempt < 3; ++attempt) {
-                float gmax = -INFINITY;
-#pragma unroll
-                for (int h = 0; h < (kMaxChunks + 3) / 4; ++h) {
-                    const int cb = c_lo + 4 * h;
-                    if (cb < c_hi) {
-                        uint32_t r[4][8];
-#pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            if (4 * h + u < kMaxChunks && cb + u < c_hi) tmem_ld_x8(s_addr + (cb + u) * 8, r[u]);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            if (4 * h + u < kMaxChunks && cb + u < c_hi)
-                                gmax = fmaxf(gmax, exp_chunk(r[u], m_s + (cb + u) * 8, scale, tail,
-                                                             (cb + u) * 8, G, gmin, p.branch_len, pk[4 * h + u]));
-                    }
-                }
+                const float gmax =
+                    !tail ? softmax_pass<0>(s_addr, c_lo, c_hi, m_s, scale, vis_s, G, gmin, pk)
+                          : softmax_pass<kTree ? 2 : 1>(s_addr, c_lo, c_hi, m_s, scale, vis_s, G, gmin, pk);
                 if (!group_any(bar_id, gmax > kGuard)) break;
 
                 // ---- a score ran past the guard: move m up to the tile maximum ----
@@ -513,7 +553,8 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
                         float s2 = __uint_as_float(r[k]) * scale;
-                        if (tail && !draft_query_sees((c8 * 8 + k) / G, gmin, p.branch_len)) s2 = -INFINITY;
+                        if (tail && (kTree ? !column_sees(vis_s[c8 * 8 + k], gmin) : (c8 * 8 + k) / G < gmin))
+                            s2 = -INFINITY;
 #pragma unroll
                         for (int o = 16; o > 0; o >>= 1)
                             s2 = fmaxf(s2, __shfl_xor_sync(0xffffffffu, s2, o));
@@ -778,8 +819,11 @@ cudaError_t launch_attn_tc(const AttnParams &p, const SeqInfo &seq, cudaStream_t
         !make_q_map(&mq, p.q, p.B, p.gamma, p.Hq, p.G))
         return cudaErrorInvalidValue;
     const size_t smem = smem_map(P.cfg).total + 1024;
-    cudaError_t err = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)smem);
+    const bool tree = p.branch_len != p.gamma;
+    cudaError_t err = tree ? cudaFuncSetAttribute(attn_tc_kernel<true>,
+                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                           : cudaFuncSetAttribute(attn_tc_kernel<false>,
+                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.n_split, p.Hkv, p.B);
@@ -791,7 +835,8 @@ cudaError_t launch_attn_tc(const AttnParams &p, const SeqInfo &seq, cudaStream_t
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = p.pdl ? 1 : 0;
-    err = cudaLaunchKernelEx(&cfg, attn_tc_kernel, P, seq, mk, mv, mq);
+    err = tree ? cudaLaunchKernelEx(&cfg, attn_tc_kernel<true>, P, seq, mk, mv, mq)
+               : cudaLaunchKernelEx(&cfg, attn_tc_kernel<false>, P, seq, mk, mv, mq);
     ++*launches;
     return err != cudaSuccess ? err : cudaGetLastError();
 }
