@@ -147,21 +147,31 @@ class ClockSampler:
 # --------------------------------------------------------------------------- #
 # reference arm: the CPU oracle, as it stands, on a bounded sample
 # --------------------------------------------------------------------------- #
+_ORACLE_INPUTS = {}
+
+
 def oracle_sample_step(cfg, sample_layers: int):
     """Times the oracle on `sample_layers` layers of attention plus the
     acceptance pass and scales the attention part to the config's layer count.
-    Returns (seconds per full step, cores used)."""
+    Returns (seconds per full step, cores used).  The sampled layers' inputs
+    are drawn once and kept: only the oracle's own work is timed."""
     import oracle
     from paper_2604_05650_b200 import workloads as W
     cores = oracle.max_threads()
     t_attn = 0.0
     mass = None
     for layer in range(sample_layers):
-        q, k, v, kv_len, span = W.attention_inputs(cfg, layer=layer)
+        key = (cfg.name, cfg.layers, layer)
+        if key not in _ORACLE_INPUTS:
+            _ORACLE_INPUTS[key] = W.attention_inputs(cfg, layer=layer)
+        q, k, v, kv_len, span = _ORACLE_INPUTS[key]
         t0 = time.perf_counter()
         _, mass = oracle.verify_attention(q, k, v, kv_len, span)
         t_attn += time.perf_counter() - t0
-    logits, draft = W.accept_inputs(cfg)
+    key = (cfg.name, "accept")
+    if key not in _ORACLE_INPUTS:
+        _ORACLE_INPUTS[key] = W.accept_inputs(cfg)
+    logits, draft = _ORACLE_INPUTS[key]
     t0 = time.perf_counter()
     oracle.loose_accept(logits, draft, mass.astype(np.float32), oracle.n_loose(cfg.lam, cfg.gamma),
                         cfg.shift_window)
@@ -173,7 +183,8 @@ def run_reference(args, cfg):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    sample_layers = 2
+    # a bounded sample per step: two layers, one when many steps are asked for
+    sample_layers = 2 if args.steps <= 30 else 1
     for _ in range(max(1, min(args.warmup, 1))):
         oracle_sample_step(cfg, 1)
     times = []
