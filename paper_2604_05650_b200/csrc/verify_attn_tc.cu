@@ -193,6 +193,14 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     const AttnParams &p = P.a;
     const TcConfig cfg = P.cfg;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // the TMA unit fetches the descriptors while everything else is set up; a warp that
+    // has nothing to do in the prologue asks for them, not the producer (whose first
+    // load is what the whole CTA waits for)
+    if (warp == kPvWarp) {
+        if (lane == 0) prefetch_tensormap(&tmap_k);
+        if (lane == 1) prefetch_tensormap(&tmap_q);
+        if (lane == 2) prefetch_tensormap(&tmap_v);
+    }
     const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
     const int L = seq.kv_len[b], vs = seq.span_start[b], ve = seq.span_end[b];
     const int M = p.M, G = p.G, gamma = p.gamma, NP = cfg.n_pad;
@@ -266,10 +274,6 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     // once; the other warps prepare shared memory and TMEM meanwhile.
     int first_k = 0, first_v = 0;   // loads issued before the CTA-wide barrier
     if (warp == 0) {
-        // the TMA unit fetches the descriptors while the barriers are set up
-        if (lane == 0) prefetch_tensormap(&tmap_k);
-        if (lane == 1) prefetch_tensormap(&tmap_v);
-        if (lane == 2) prefetch_tensormap(&tmap_q);
         {
             // one barrier per lane, all at once (an mbarrier.init costs about a hundred
             // cycles): barriers sit in the order k_full, k_empty, v_full, v_empty,
@@ -291,13 +295,15 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         if (lane == 0) {
             // inputs may come from the kernel before this one in the stream
             grid_dependency_wait();
+            // the first K tile comes from HBM and is needed first: it goes out before Q
+            first_k = min(T, cfg.ks);
+            first_v = min(T, cfg.vs);
+            load_k(0);
             mbar_arrive_expect_tx(q_full, (uint32_t)M * 256u);
             tma_load_4d(base + sm.q, &tmap_q, q_full, 0, kvh * G, 0, b);
             tma_load_4d(base + sm.q + NP * 128, &tmap_q, q_full, 64, kvh * G, 0, b);
-            first_k = min(T, cfg.ks);
-            first_v = min(T, cfg.vs);
             for (int i = 0; i < first_v; ++i) {
-                if (i < first_k) load_k(i);
+                if (i > 0 && i < first_k) load_k(i);
                 load_v(i);
             }
         }
