@@ -195,27 +195,44 @@ attn_simt_kernel(const AttnParams p, const SeqInfo seq)
 }
 
 // Merge of the KV splits: one warp per (sequence, KV head, row), each lane four
-// output channels.  Splits are merged in index order, so the result does not
-// depend on scheduling.  The kernel may be launched programmatically dependent
-// on the attention kernel: it lets the next launch be scheduled, then waits
-// for the partials.
+// output channels.  The result does not depend on scheduling (every sum has a fixed
+// order).  The kernel may be launched programmatically dependent on the attention
+// kernel: it lets the next launch be scheduled, then waits for the partials.
 //
-// Batches of 32 splits: lane u fetches the statistics of split u while every
-// lane fetches its four channels of all 32 partial outputs, so a batch costs
-// one round trip to L2.  The running reference exponent moves up between
-// batches like an online softmax.
+// The kernel runs once per layer on cold instruction caches, where straight-line code
+// costs about ten cycles per instruction: so the splits' rows come in by cp.async in a
+// short rolled loop (a batch of up to 32 splits per round trip to L2, landing in shared
+// memory), lane u meanwhile turns the statistics of split u into its weight, and a second
+// rolled loop accumulates from shared memory.  The running reference exponent moves up
+// between batches like an online softmax.
 constexpr int kCombineBatch = 32;
 constexpr int kCombineWarps = 2;
 
-__global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const AttnParams p)
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
 {
+    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ float warp_sum(float x)
+{
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+    return x;
+}
+
+// dynamic shared memory per warp: `batch` rows of 32 float4, then `batch` weights
+__global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const AttnParams p, const int batch)
+{
+    extern __shared__ float4 combine_smem[];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int lane = threadIdx.x & 31;
-    const int r = blockIdx.x * kCombineWarps + (threadIdx.x >> 5), kvh = blockIdx.y, b = blockIdx.z;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int r = blockIdx.x * kCombineWarps + w, kvh = blockIdx.y, b = blockIdx.z;
     const int M = p.M, D = p.D, ns = p.n_split;
     if (r >= M) return;
     const bool active = lane * 4 < D;                   // D = 64 uses half the lanes
+    float4 *rows = combine_smem + (size_t)w * (batch * 32 + (batch + 3) / 4);
+    float *weights = reinterpret_cast<float *>(rows + batch * 32);
     const size_t unit0 = ((size_t)b * p.Hkv + kvh) * ns;
     const float4 *ps = reinterpret_cast<const float4 *>(p.part_stat) + unit0 * (size_t)M + r;
     const float4 *po = reinterpret_cast<const float4 *>(p.part_o + (unit0 * (size_t)M + r) * D) +
@@ -224,12 +241,14 @@ __global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const 
 
     float m_run = -INFINITY, l = 0.f, lv = 0.f;
     float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s0 = 0; s0 < ns; s0 += kCombineBatch) {
-        const int n = min(kCombineBatch, ns - s0);
-        float4 v[kCombineBatch];
-#pragma unroll
-        for (int u = 0; u < kCombineBatch; ++u)
-            v[u] = u < n ? __ldcg(po + (size_t)(s0 + u) * o_stride) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s0 = 0; s0 < ns; s0 += batch) {
+        const int n = min(batch, ns - s0);
+        if (active) {
+            const float4 *src = po + (size_t)s0 * o_stride;
+            float4 *dst = rows + lane;
+            for (int u = 0; u < n; ++u, src += o_stride, dst += 32) cp_async16(dst, src);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
         float4 st = make_float4(-INFINITY, 0.f, 0.f, 0.f);
         if (lane < n) st = __ldcg(ps + (size_t)(s0 + lane) * M);
         float m_b = st.y > 0.f ? st.x : -INFINITY;
@@ -242,20 +261,24 @@ __global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const 
             m_run = m_b;
         }
         const float w_mine = st.y > 0.f ? exp2f(st.x - m_run) : 0.f;
-#pragma unroll
-        for (int u = 0; u < kCombineBatch; ++u) {
-            if (u < n) {
-                const float w = __shfl_sync(0xffffffffu, w_mine, u);
-                const float lu = __shfl_sync(0xffffffffu, st.y, u);
-                const float lvu = __shfl_sync(0xffffffffu, st.z, u);
-                l = fmaf(w, lu, l);
-                lv = fmaf(w, lvu, lv);
-                o.x = fmaf(w, v[u].x, o.x);
-                o.y = fmaf(w, v[u].y, o.y);
-                o.z = fmaf(w, v[u].z, o.z);
-                o.w = fmaf(w, v[u].w, o.w);
+        l += warp_sum(w_mine * st.y);
+        lv += warp_sum(w_mine * st.z);
+        if (lane < n) weights[lane] = w_mine;           // batch <= 32: one weight per lane
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncwarp();
+        if (active) {
+            const float4 *v = rows + lane;
+#pragma unroll 2
+            for (int u = 0; u < n; ++u, v += 32) {
+                const float wu = weights[u];
+                const float4 x = *v;
+                o.x = fmaf(wu, x.x, o.x);
+                o.y = fmaf(wu, x.y, o.y);
+                o.z = fmaf(wu, x.z, o.z);
+                o.w = fmaf(wu, x.w, o.w);
             }
         }
+        __syncwarp();
     }
     const float inv = 1.f / l;
     const int g = r / p.G, hg = r - g * p.G;
@@ -307,7 +330,9 @@ cudaError_t launch_attn_combine(const AttnParams &p, cudaStream_t stream, int *l
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = p.pdl ? 1 : 0;
-    cudaError_t err = cudaLaunchKernelEx(&cfg, attn_combine_kernel, p);
+    const int batch = p.n_split < kCombineBatch ? p.n_split : kCombineBatch;
+    cfg.dynamicSmemBytes = (size_t)kCombineWarps * (batch * 32 + (batch + 3) / 4) * sizeof(float4);
+    cudaError_t err = cudaLaunchKernelEx(&cfg, attn_combine_kernel, p, batch);
     ++*launches;
     return err != cudaSuccess ? err : cudaGetLastError();
 }
