@@ -213,19 +213,14 @@ __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
     const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
 }
-__device__ __forceinline__ float warp_sum(float x)
-{
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
-    return x;
-}
 
 // dynamic shared memory per warp: `batch` rows of 32 float4, then `batch` weights
 __global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const AttnParams p, const int batch)
 {
     extern __shared__ float4 combine_smem[];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // every address is worked out before the wait for the attention grid: the CTA is
+    // resident by then, and the cold parameter loads and index arithmetic cost it nothing
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int r = blockIdx.x * kCombineWarps + w, kvh = blockIdx.y, b = blockIdx.z;
     const int M = p.M, D = p.D, ns = p.n_split;
@@ -238,19 +233,25 @@ __global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const 
     const float4 *po = reinterpret_cast<const float4 *>(p.part_o + (unit0 * (size_t)M + r) * D) +
                        (active ? lane : 0);
     const size_t o_stride = (size_t)M * D / 4;          // float4 units between splits
+    const int g = r / p.G, hg = r - g * p.G;
+    const size_t row = ((size_t)b * p.gamma + g) * p.Hq + kvh * p.G + hg;
+    uint16_t *out_row = p.out + row * D + lane * 4;
+    float *mass_row = p.mass + row;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     float m_run = -INFINITY, l = 0.f, lv = 0.f;
     float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int s0 = 0; s0 < ns; s0 += batch) {
         const int n = min(batch, ns - s0);
+        // the statistics first: the weights hang on them, the rows are only needed after
+        float4 st = make_float4(-INFINITY, 0.f, 0.f, 0.f);
+        if (lane < n) st = __ldcg(ps + (size_t)(s0 + lane) * M);
         if (active) {
             const float4 *src = po + (size_t)s0 * o_stride;
             float4 *dst = rows + lane;
             for (int u = 0; u < n; ++u, src += o_stride, dst += 32) cp_async16(dst, src);
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
-        float4 st = make_float4(-INFINITY, 0.f, 0.f, 0.f);
-        if (lane < n) st = __ldcg(ps + (size_t)(s0 + lane) * M);
         float m_b = st.y > 0.f ? st.x : -INFINITY;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) m_b = fmaxf(m_b, __shfl_xor_sync(0xffffffffu, m_b, off));
@@ -261,14 +262,20 @@ __global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const 
             m_run = m_b;
         }
         const float w_mine = st.y > 0.f ? exp2f(st.x - m_run) : 0.f;
-        l += warp_sum(w_mine * st.y);
-        lv += warp_sum(w_mine * st.z);
+        float sl = w_mine * st.y, slv = w_mine * st.z;   // two sums, one butterfly
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            sl += __shfl_xor_sync(0xffffffffu, sl, off);
+            slv += __shfl_xor_sync(0xffffffffu, slv, off);
+        }
+        l += sl;
+        lv += slv;
         if (lane < n) weights[lane] = w_mine;           // batch <= 32: one weight per lane
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         __syncwarp();
         if (active) {
             const float4 *v = rows + lane;
-#pragma unroll 2
+#pragma unroll 3
             for (int u = 0; u < n; ++u, v += 32) {
                 const float wu = weights[u];
                 const float4 x = *v;
@@ -281,17 +288,15 @@ __global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const 
         __syncwarp();
     }
     const float inv = 1.f / l;
-    const int g = r / p.G, hg = r - g * p.G;
-    const size_t row = ((size_t)b * p.gamma + g) * p.Hq + kvh * p.G + hg;
     if (active) {
         __nv_bfloat162 lo = __floats2bfloat162_rn(o.x * inv, o.y * inv);
         __nv_bfloat162 hi = __floats2bfloat162_rn(o.z * inv, o.w * inv);
         uint2 pk;
         pk.x = *reinterpret_cast<uint32_t *>(&lo);
         pk.y = *reinterpret_cast<uint32_t *>(&hi);
-        *reinterpret_cast<uint2 *>(p.out + row * D + lane * 4) = pk;
+        *reinterpret_cast<uint2 *>(out_row) = pk;
     }
-    if (lane == 0) p.mass[row] = lv * inv;
+    if (lane == 0) *mass_row = lv * inv;
 }
 
 }  // namespace

@@ -684,37 +684,41 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 }
             }
         } else {
-            // partial O^T: up to four chunks of 8 columns in flight per wait
-            for (int cb = c_lo; cb < c_hi; cb += 4) {
-                uint32_t r[4][8];
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (cb + u < c_hi) tmem_ld_x8(tm_o + lane_addr + (cb + u) * 8, r[u]);
+            // This code runs once, on cold instruction caches, where every instruction
+            // costs about ten cycles: short rolled loops, one chunk of 8 columns a turn;
+            // only a last chunk that is not full takes the guarded path.
+            float *po = part_o + (size_t)c_lo * 8 * 128 + row;
+#pragma unroll 1
+            for (int c8 = c_lo; c8 < c_hi; ++c8, po += 8 * 128) {
+                uint32_t r[8];
+                tmem_ld_x8(tm_o + lane_addr + c8 * 8, r);
                 tmem_wait_ld();
+                if (c8 * 8 + 8 <= M) {
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    if (cb + u < c_hi) {
+                    for (int k = 0; k < 8; ++k) po[k * 128] = __uint_as_float(r[k]);
+                } else {
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            const int n = (cb + u) * 8 + k;
-                            if (n < M) part_o[(size_t)n * 128 + row] = __uint_as_float(r[u][k]);
-                        }
-                    }
+                    for (int k = 0; k < 8; ++k)
+                        if (c8 * 8 + k < M) po[k * 128] = __uint_as_float(r[k]);
                 }
             }
             if (wq == 0) {
+#pragma unroll 1
                 for (int c8 = c_lo; c8 < c_hi; ++c8) {
                     uint32_t r[8];
                     tmem_ld_x8(tm_l + c8 * 8, r);     // lane 0: l, lane 1: l_vis
                     tmem_wait_ld();
+                    // lane k takes column k of the chunk: l from lane 0, l_vis from lane 1
+                    float lk = 0.f, lvk = 0.f;
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
-                        const int n = c8 * 8 + k;
-                        const float lv = __shfl_sync(0xffffffffu, __uint_as_float(r[k]), 1);
-                        if (lane == 0 && n < M)
-                            *reinterpret_cast<float4 *>(part_stat + n * 4) =
-                                make_float4(m_s[n], __uint_as_float(r[k]), lv, 0.f);
+                        const float a = __shfl_sync(0xffffffffu, __uint_as_float(r[k]), 0);
+                        const float c = __shfl_sync(0xffffffffu, __uint_as_float(r[k]), 1);
+                        if (lane == k) { lk = a; lvk = c; }
                     }
+                    if (lane < 8 && c8 * 8 + lane < M)
+                        *reinterpret_cast<float4 *>(part_stat + (c8 * 8 + lane) * 4) =
+                            make_float4(m_s[c8 * 8 + lane], lk, lvk, 0.f);
                 }
             }
         }
