@@ -412,7 +412,8 @@ def run_ours(args, cfg):
             "cuda_graph": graph_attn is not None, "roofline": roofline, "clocks": clocks.summary()}
 
     if not args.no_next_rows and world == 1:
-        line["next_rows"] = {"visual_relevance": time_visual_relevance(cfg, ctx, stream, torch, dev, peak)}
+        line["next_rows"] = {"visual_relevance": time_visual_relevance(cfg, ctx, stream, torch, dev, peak),
+                             "paged_attention": time_paged_attention(cfg, ctx, stream, ks, vs_, qs, torch, dev, peak)}
 
     # end to end through the host-buffer entry points
     if not args.no_e2e:
@@ -462,6 +463,67 @@ def time_visual_relevance(cfg, ctx, stream, torch, dev, peak):
     gbs = nbytes / (us * 1e-6) / 1e9
     return {"us_per_call": us, "n_visual": lv, "dim": d, "top_n": 10, "bytes_per_call": nbytes,
             "achieved_gbs": gbs, "frac_of_peak": gbs / peak, "launches_per_call": 3}
+
+
+def time_paged_attention(cfg, ctx, stream, ks, vs_, qs, torch, dev, peak):
+    """The verify attention on a paged cache (512-position pages scattered at random
+    over a pool): the first layers' caches of the step, re-read as page pools, in a
+    graph of up to eight layers (each streams its own 134 MB, more than L2 together)."""
+    from paper_2604_05650_b200 import binding
+    B, g, Hq, Hkv, D, L = cfg.batch, cfg.gamma, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.kv_len
+    page = 512
+    if L % page or D != 128:
+        return None
+    n_layers = min(8, len(ks))
+    per_seq = L // page
+    n_pages = B * per_seq
+    # [B, Hkv, L, D] -> [B * L / page, Hkv, page, D]: logical page j of sequence b sits at
+    # pool page b * per_seq + j; then the pool pages are shuffled and the table follows
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(cfg.seed + 99)
+    perm = torch.randperm(n_pages, generator=gen)
+    inv = torch.empty_like(perm)
+    inv[perm] = torch.arange(n_pages)
+    pools = []
+    for l in range(n_layers):
+        pk = ks[l].view(B, Hkv, per_seq, page, D).permute(0, 2, 1, 3, 4).reshape(n_pages, Hkv, page, D)
+        pv = vs_[l].view(B, Hkv, per_seq, page, D).permute(0, 2, 1, 3, 4).reshape(n_pages, Hkv, page, D)
+        pools.append((pk[perm.to(dev)].contiguous(), pv[perm.to(dev)].contiguous()))
+    table = inv.view(B, per_seq).to(torch.int32).to(dev)
+    out = torch.empty((B, g, Hq, D), dtype=torch.bfloat16, device=dev)
+    mass = torch.empty((B, g, Hq), dtype=torch.float32, device=dev)
+    shape = binding.attn_shape(B, g, Hq, Hkv, D, L, 0, 0)
+    kv_len = np.full((B,), L, dtype=np.int32)
+    span = np.tile(np.asarray([cfg.span], dtype=np.int32), (B, 1))
+
+    def layers():
+        for l in range(n_layers):
+            ctx.verify_attention_paged(shape, page, n_pages, qs[l], pools[l][0], pools[l][1], table,
+                                       kv_len, span, out, mass)
+
+    with torch.cuda.stream(stream):
+        layers()
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            ctx.set_stream(torch.cuda.current_stream().cuda_stream)
+            layers()
+        ctx.set_stream(stream.cuda_stream)
+        for _ in range(3):
+            graph.replay()
+        reps = 10
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            graph.replay()
+        e1.record(stream)
+    stream.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / (reps * n_layers)
+    nbytes = cfg.kv_bytes_per_layer + 2 * B * g * Hq * D * 2 + B * g * Hq * 4
+    gbs = nbytes / (us * 1e-6) / 1e9
+    del pools
+    return {"us_per_layer": us, "page_size": page, "n_pages": n_pages, "layers_in_graph": n_layers,
+            "bytes_per_layer": nbytes, "achieved_gbs": gbs, "frac_of_peak": gbs / peak}
 
 
 def run_e2e(args, cfg, ctx, stream, qs, ks, vs_, logits, draft, torch, dev, world, barrier, dist):

@@ -197,6 +197,30 @@ lvspec_status_t lvspec_verify_attention_tree(lvspec_ctx_t *ctx, const lvspec_att
 lvspec_status_t lvspec_select_branch(lvspec_ctx_t *ctx, int32_t batch, int32_t n_branches,
                                      const int32_t *accept_len, int32_t *best_branch, int32_t *best_len);
 
+/* lvspec_verify_attention on a PAGED cache (a serving engine's layout; the paper's
+ * runs keep one contiguous cache per sequence, Sec. "Experimental Setup", so this is a
+ * layout variant of Eq. 1, not another operation).  K and V live in pools of
+ * fixed-size pages shared by all sequences:
+ *
+ *   k_pool, v_pool  device, bf16  [n_pages, Hkv, page_size, D]
+ *   block_table     device, int32 [B, kv_capacity / page_size]: pool page of each
+ *                   logical page of a sequence; logical position j of sequence b
+ *                   is row j % page_size of page block_table[b][j / page_size]
+ *
+ * shape->kv_capacity is the logical capacity per sequence, a whole number of
+ * pages; page_size is a multiple of 128 (one tile never straddles pages).  Only
+ * the entries of pages that hold positions below kv_len[b] are read; an entry
+ * outside 0..n_pages-1 is not an error: its positions read as zeros.  The block
+ * table is read on the device during the call (it may be written by the kernel
+ * before this call in the stream).  All else is as for lvspec_verify_attention:
+ * same arithmetic, same results bit for bit as on the equivalent contiguous cache.
+ * UNSUPPORTED for head_dim other than 128 and for LVSPEC_KERNEL_SIMT. */
+lvspec_status_t lvspec_verify_attention_paged(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                              int32_t page_size, int32_t n_pages, const void *q,
+                                              const void *k_pool, const void *v_pool,
+                                              const int32_t *block_table, const int32_t *kv_len,
+                                              const int32_t *visual_span, void *out, float *visual_mass);
+
 /* Same operation on HOST buffers: copies q, the caches, and the results through
  * device staging memory the context owns (grown on demand), on the context's
  * stream, and synchronises before returning.  All seven arrays are host

@@ -30,7 +30,7 @@ EXPORTS = (
     "lvspec_loose_accept", "lvspec_loose_accept_ex", "lvspec_loose_accept_host",
     "lvspec_loose_accept_static", "lvspec_row_inv_norms", "lvspec_visual_relevance",
     "lvspec_selftest_wait_expiry", "lvspec_loose_accept_emit",
-    "lvspec_verify_attention_tree", "lvspec_select_branch",
+    "lvspec_verify_attention_tree", "lvspec_select_branch", "lvspec_verify_attention_paged",
 )
 
 
@@ -87,6 +87,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lvspec_selftest_wait_expiry.argtypes = [vp, i32]
     lib.lvspec_verify_attention_tree.argtypes = [vp, S, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.lvspec_select_branch.argtypes = [vp, i32, i32, vp, vp, vp]
+    lib.lvspec_verify_attention_paged.argtypes = [vp, S, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.lvspec_loose_accept_emit.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp, vp, vp, vp, vp]
     lib.lvspec_row_inv_norms.argtypes = [vp, ctypes.c_int64, i32, vp, vp]
     lib.lvspec_visual_relevance.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, i32, vp]
@@ -187,6 +188,18 @@ class Context:
         self._check(self._lib.lvspec_verify_attention_tree(
             self._h, ctypes.byref(shape), int(n_branches), _addr(q), _addr(k_cache), _addr(v_cache),
             kv_len.ctypes.data, span.ctypes.data, _addr(out), _addr(visual_mass)))
+
+    def verify_attention_paged(self, shape: AttnShape, page_size, n_pages, q, k_pool, v_pool, block_table,
+                               kv_len, visual_span, out, visual_mass) -> None:
+        """k_pool / v_pool: device [n_pages, Hkv, page_size, D]; block_table: device int32
+        [B, kv_capacity / page_size]; kv_len, visual_span: host."""
+        kv_len, span = _i32(kv_len), _i32(visual_span)
+        if shape.batch >= 1 and (kv_len.size != shape.batch or span.size != 2 * shape.batch):
+            raise ValueError("kv_len needs B entries and visual_span B pairs")
+        self._check(self._lib.lvspec_verify_attention_paged(
+            self._h, ctypes.byref(shape), int(page_size), int(n_pages), _addr(q), _addr(k_pool),
+            _addr(v_pool), _addr(block_table), kv_len.ctypes.data, span.ctypes.data, _addr(out),
+            _addr(visual_mass)))
 
     def select_branch(self, batch, n_branches, accept_len, best_branch, best_len) -> None:
         self._check(self._lib.lvspec_select_branch(self._h, int(batch), int(n_branches), _addr(accept_len),

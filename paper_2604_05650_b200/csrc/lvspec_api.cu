@@ -148,9 +148,14 @@ lvspec_status_t check_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, c
     return LVSPEC_OK;
 }
 
+struct PagedCache {          // page pools instead of one contiguous cache per sequence
+    const int32_t *block_table = nullptr;
+    int page_size = 0, pages_per_seq = 0, n_pages = 0;
+};
+
 lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, const SeqInfo &seq,
                               int max_len, const void *q, const void *k, const void *v, void *out,
-                              float *mass, int branch_len = 0)
+                              float *mass, int branch_len = 0, const PagedCache *paged = nullptr)
 {
     AttnParams p;
     std::memset(&p, 0, sizeof p);
@@ -172,6 +177,12 @@ lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, con
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)p.D));
     p.pdl = ctx->pdl ? 1 : 0;
     p.branch_len = branch_len > 0 ? branch_len : p.gamma;
+    if (paged) {
+        p.block_table = paged->block_table;
+        p.page_size = paged->page_size;
+        p.pages_per_seq = paged->pages_per_seq;
+        p.n_pages = paged->n_pages;
+    }
 
     const size_t o_bytes = part_o_elems(p) * sizeof(float);
     const size_t st_bytes = part_stat_elems(p) * sizeof(float);
@@ -435,6 +446,39 @@ lvspec_status_t lvspec_verify_attention_tree(lvspec_ctx_t *ctx, const lvspec_att
     if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
     return run_attention(ctx, shape, seq, max_len, q, k_cache, v_cache, out, visual_mass,
                          shape->gamma / n_branches);
+}
+
+lvspec_status_t lvspec_verify_attention_paged(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                              int32_t page_size, int32_t n_pages, const void *q,
+                                              const void *k_pool, const void *v_pool,
+                                              const int32_t *block_table, const int32_t *kv_len,
+                                              const int32_t *visual_span, void *out, float *visual_mass)
+{
+    SeqInfo seq;
+    int max_len = 0;
+    lvspec_status_t st = check_attention(ctx, shape, q, k_pool, v_pool, kv_len, visual_span, out,
+                                         visual_mass, true, &seq, &max_len);
+    if (st != LVSPEC_OK) return st;
+    if (!block_table || (reinterpret_cast<uintptr_t>(block_table) & 3u))
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "block_table is null or misaligned");
+    if (page_size < 128 || page_size % 128 != 0)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "page_size must be a positive multiple of 128");
+    if (n_pages < 1 || (long long)n_pages * shape->n_kv_heads > 2147483647ll)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "n_pages outside 1..2^31 / n_kv_heads");
+    if (shape->kv_capacity % page_size != 0)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "kv_capacity must be a whole number of pages");
+    if (shape->head_dim != 128 || shape->kernel == LVSPEC_KERNEL_SIMT)
+        return fail(ctx, LVSPEC_ERR_UNSUPPORTED, "the paged cache needs the tcgen05 kernel (head_dim 128)");
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
+    PagedCache pc;
+    pc.block_table = block_table;
+    pc.page_size = page_size;
+    pc.pages_per_seq = shape->kv_capacity / page_size;
+    pc.n_pages = n_pages;
+    lvspec_attn_shape_t s = *shape;
+    s.kernel = LVSPEC_KERNEL_TCGEN05;
+    return run_attention(ctx, &s, seq, max_len, q, k_pool, v_pool, out, visual_mass, 0, &pc);
 }
 
 lvspec_status_t lvspec_verify_attention_host(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,

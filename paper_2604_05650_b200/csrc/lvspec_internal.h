@@ -27,6 +27,10 @@ struct AttnParams {
     int32_t B, gamma, Hq, Hkv, D, Lmax, G, M, n_split;
     int32_t pdl;           // launch programmatically dependent on the previous kernel
     int32_t branch_len;    // draft tokens per tree branch (= gamma for a plain chain)
+    // Paged cache (page_size > 0): k and v are pools [n_pages, Hkv, page_size, D]; logical
+    // page j of sequence b is pool page block_table[b * pages_per_seq + j]
+    const int32_t *block_table;
+    int32_t page_size, pages_per_seq, n_pages;
     float scale_log2;      // log2(e) / sqrt(D)
 };
 

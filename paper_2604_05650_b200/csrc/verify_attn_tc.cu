@@ -57,11 +57,12 @@ struct TcConfig {
     int n_pad;   // MMA N: rows padded to a multiple of 16
     int ks, vs, pb;   // K slots, V slots, P buffers
     int tmem_cols;
+    int page_slots;   // paged cache: pool pages of this split's tiles, one entry per tile
 };
 
 // Byte offsets of the shared-memory regions (relative to a 1024-aligned base).
 struct SmemMap {
-    uint32_t k, v, q, p, a2, m, dl, tmx, vis, bars, misc, total;
+    uint32_t k, v, q, p, a2, m, dl, tmx, vis, bars, misc, pages, total;
 };
 __host__ __device__ inline SmemMap smem_map(const TcConfig &c)
 {
@@ -78,6 +79,7 @@ __host__ __device__ inline SmemMap smem_map(const TcConfig &c)
     s.vis = o;  o += c.n_pad * 8;
     s.bars = o; o += 8 * (2 * c.ks + 2 * c.vs + 4 + 2 * c.pb + 3);
     s.misc = o; o += 16;
+    s.pages = o; o += 4 * c.page_slots;
     s.total = o;
     return s;
 }
@@ -183,8 +185,9 @@ __device__ __forceinline__ float softmax_pass(uint32_t s_addr, int c_lo, int c_h
 }
 
 // kTree: the draft slots hold several branches (the visibility table is only built
-// and read then; the plain chain keeps its arithmetic mask)
-template <bool kTree>
+// and read then; the plain chain keeps its arithmetic mask).  kPaged: K and V are page
+// pools and a tile's position in them comes from the sequence's block table.
+template <bool kTree, bool kPaged>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUtensorMap tmap_k,
                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_q)
@@ -254,18 +257,33 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
 
     // the cache is read once per call: it should not push the split partials out of L2
     const uint64_t stream_policy = l2_evict_first_policy();
+    // where tile i of this split sits: (position, row of the [.., positions, 128] map)
+    volatile int32_t *page_s = reinterpret_cast<volatile int32_t *>(gbase + sm.pages);
+    auto tile_at = [&](int i, int &pos0, int &map_row) {
+        pos0 = (t_begin + i) * kTilePos;
+        map_row = bh;
+        if (kPaged) {
+            // a page holds a whole number of tiles; an entry outside the pool reads as zeros
+            pos0 -= (pos0 / p.page_size) * p.page_size;
+            map_row = page_s[i] * p.Hkv + kvh;
+        }
+    };
     auto load_k = [&](int i) {
-        const int ks = i % cfg.ks, pos0 = (t_begin + i) * kTilePos;
+        const int ks = i % cfg.ks;
+        int pos0, map_row;
+        tile_at(i, pos0, map_row);
         mbar_arrive_expect_tx(k_full(ks), kSlotBytes);
-        tma_load_3d_hint(base + sm.k + ks * kSlotBytes, &tmap_k, k_full(ks), 0, pos0, bh, stream_policy);
-        tma_load_3d_hint(base + sm.k + ks * kSlotBytes + kBoxBytes, &tmap_k, k_full(ks), 64, pos0, bh,
+        tma_load_3d_hint(base + sm.k + ks * kSlotBytes, &tmap_k, k_full(ks), 0, pos0, map_row, stream_policy);
+        tma_load_3d_hint(base + sm.k + ks * kSlotBytes + kBoxBytes, &tmap_k, k_full(ks), 64, pos0, map_row,
                          stream_policy);
     };
     auto load_v = [&](int i) {
-        const int vsl = i % cfg.vs, pos0 = (t_begin + i) * kTilePos;
+        const int vsl = i % cfg.vs;
+        int pos0, map_row;
+        tile_at(i, pos0, map_row);
         mbar_arrive_expect_tx(v_full(vsl), kSlotBytes);
-        tma_load_3d_hint(base + sm.v + vsl * kSlotBytes, &tmap_v, v_full(vsl), 0, pos0, bh, stream_policy);
-        tma_load_3d_hint(base + sm.v + vsl * kSlotBytes + kBoxBytes, &tmap_v, v_full(vsl), 64, pos0, bh,
+        tma_load_3d_hint(base + sm.v + vsl * kSlotBytes, &tmap_v, v_full(vsl), 0, pos0, map_row, stream_policy);
+        tma_load_3d_hint(base + sm.v + vsl * kSlotBytes + kBoxBytes, &tmap_v, v_full(vsl), 64, pos0, map_row,
                          stream_policy);
     };
 
@@ -292,6 +310,14 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             fence_proxy_async_smem();
         }
         __syncwarp();
+        if (kPaged) {
+            // the block table too may come from the kernel before this one: the warp reads
+            // this split's entries (one per tile) after the wait, then lane 0 goes on
+            grid_dependency_wait();
+            const int32_t *row = p.block_table + (size_t)b * p.pages_per_seq;
+            for (int i = lane; i < T; i += 32) page_s[i] = __ldg(row + ((t_begin + i) * kTilePos) / p.page_size);
+            __syncwarp();
+        }
         if (lane == 0) {
             // inputs may come from the kernel before this one in the stream
             grid_dependency_wait();
@@ -795,10 +821,11 @@ bool make_q_map(CUtensorMap *map, const void *ptr, int B, int gamma, int Hq, int
 
 constexpr uint32_t kMaxSmem = 232448 - 1024;   // 227 KB less the alignment slack
 
-TcConfig pick_config(int M)
+TcConfig pick_config(int M, int page_slots)
 {
     TcConfig c;
     c.n_pad = (M + 15) & ~15;
+    c.page_slots = page_slots;
     // deepest K/V rings that fit: bytes in flight matter more than a second P buffer,
     // since the probabilities wait in registers for the buffer anyway
     const int tries[6][3] = {{3, 3, 2}, {3, 3, 1}, {2, 3, 2}, {2, 3, 1}, {2, 2, 2}, {2, 2, 1}};
@@ -823,17 +850,23 @@ cudaError_t launch_attn_tc(const AttnParams &p, const SeqInfo &seq, cudaStream_t
 {
     TcParams P;
     P.a = p;
-    P.cfg = pick_config(p.M);
+    const bool paged = p.page_size > 0;
+    // paged: one block-table entry per tile of the longest split, rounded up to 4
+    const int tiles = (p.Lmax + kTilePos - 1) / kTilePos;
+    P.cfg = pick_config(p.M, paged ? ((tiles + p.n_split - 1) / p.n_split + 4) & ~3 : 0);
+    if (smem_map(P.cfg).total > kMaxSmem) return cudaErrorInvalidConfiguration;
     CUtensorMap mk, mv, mq;
-    if (!make_kv_map(&mk, p.k, p.Lmax, p.B * p.Hkv) || !make_kv_map(&mv, p.v, p.Lmax, p.B * p.Hkv) ||
+    const int map_len = paged ? p.page_size : p.Lmax;
+    const int map_rows = paged ? p.n_pages * p.Hkv : p.B * p.Hkv;
+    if (!make_kv_map(&mk, p.k, map_len, map_rows) || !make_kv_map(&mv, p.v, map_len, map_rows) ||
         !make_q_map(&mq, p.q, p.B, p.gamma, p.Hq, p.G))
         return cudaErrorInvalidValue;
     const size_t smem = smem_map(P.cfg).total + 1024;
     const bool tree = p.branch_len != p.gamma;
-    cudaError_t err = tree ? cudaFuncSetAttribute(attn_tc_kernel<true>,
-                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-                           : cudaFuncSetAttribute(attn_tc_kernel<false>,
-                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (tree && paged) return cudaErrorNotSupported;
+    auto kernel = paged ? attn_tc_kernel<false, true>
+                        : (tree ? attn_tc_kernel<true, false> : attn_tc_kernel<false, false>);
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.n_split, p.Hkv, p.B);
@@ -845,8 +878,7 @@ cudaError_t launch_attn_tc(const AttnParams &p, const SeqInfo &seq, cudaStream_t
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = p.pdl ? 1 : 0;
-    err = tree ? cudaLaunchKernelEx(&cfg, attn_tc_kernel<true>, P, seq, mk, mv, mq)
-               : cudaLaunchKernelEx(&cfg, attn_tc_kernel<false>, P, seq, mk, mv, mq);
+    err = cudaLaunchKernelEx(&cfg, kernel, P, seq, mk, mv, mq);
     ++*launches;
     return err != cudaSuccess ? err : cudaGetLastError();
 }
