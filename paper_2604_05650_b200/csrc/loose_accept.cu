@@ -107,21 +107,37 @@ __global__ void __launch_bounds__(kThreads) loose_accept_kernel(const AcceptPara
     __shared__ int draft_s[LVSPEC_MAX_GAMMA];
     __shared__ double score_s[LVSPEC_MAX_GAMMA];
     __shared__ unsigned char acc_s[LVSPEC_MAX_GAMMA];
-    if (tid < gamma) {
-        const size_t rid = (size_t)b * gamma + tid;
-        const volatile float *pv = p.part_val + rid * p.n_vsplit;
-        const volatile int *pi = p.part_idx + rid * p.n_vsplit;
+    // One warp per position (round robin): the lanes fetch the slices' partials and the
+    // heads' masses side by side, so a position costs one round trip to L2, not one per
+    // partial.  "Greater value, then lower index" is a total order: any reduction tree
+    // gives the same winner.  The masses are added in index order, in double, as the rule
+    // is defined: lane order restored by shuffles.
+    for (int i = warp; i < gamma; i += kThreads / 32) {
+        const size_t rid = (size_t)b * gamma + i;
         Best bb = {-INFINITY, kNoIndex};
-        for (int s = 0; s < p.n_vsplit; ++s) {
-            Best o = {pv[s], pi[s]};
+        for (int s = lane; s < p.n_vsplit; s += 32) {
+            Best o = {__ldcg(p.part_val + rid * p.n_vsplit + s), __ldcg(p.part_idx + rid * p.n_vsplit + s)};
             bb = better(bb, o);
         }
-        y_s[tid] = (bb.i == kNoIndex) ? 0 : bb.i;   // nothing above -inf: token 0
-        draft_s[tid] = p.draft[rid];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            Best other;
+            other.v = __shfl_xor_sync(0xffffffffu, bb.v, o);
+            other.i = __shfl_xor_sync(0xffffffffu, bb.i, o);
+            bb = better(bb, other);
+        }
         double sc = 0.0;
         const float *mrow = p.mass + rid * p.Hm;
-        for (int h = 0; h < p.Hm; ++h) sc += (double)mrow[h];
-        score_s[tid] = sc;
+        for (int h0 = 0; h0 < p.Hm; h0 += 32) {
+            const float mine = h0 + lane < p.Hm ? mrow[h0 + lane] : 0.f;
+            const int n = min(32, p.Hm - h0);
+            for (int h = 0; h < n; ++h) sc += (double)__shfl_sync(0xffffffffu, mine, h);
+        }
+        if (lane == 0) {
+            y_s[i] = (bb.i == kNoIndex) ? 0 : bb.i;   // nothing above -inf: token 0
+            draft_s[i] = p.draft[rid];
+            score_s[i] = sc;
+        }
     }
     __syncthreads();
     if (tid < gamma) {
