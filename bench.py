@@ -373,7 +373,8 @@ def run_ours(args, cfg):
     clocks.stop()
     status = ctx.device_status()
     ms_total = ev0.elapsed_time(ev1)
-    ms_attn = sum(a.elapsed_time(b) for a, b in attn_ev) / args.steps
+    attn_ms = sorted(a.elapsed_time(b) for a, b in attn_ev)
+    ms_attn = sum(attn_ms) / args.steps
     ms_total_max = slowest_rank_ms(ms_total, world, dist, dev)
     ms_step = ms_total_max / args.steps
     value = whole_job_tokens_per_s(world, B, g, ms_step)
@@ -397,10 +398,24 @@ def run_ours(args, cfg):
         src = os.path.join(ROOT, tr.get("kernel_source", ""))
         if os.path.exists(src) and hashlib.sha256(open(src, "rb").read()).hexdigest() == tr.get("kernel_source_sha256"):
             traffic = tr.get(f"config{cfg_id_of(cfg)}")
+    # secondary bounds of the same launch: useful tensor flops (two products, 2 flops per
+    # multiply-add) against the measured bf16 GEMM rate, and exponentials against the
+    # special-function rate (16 per clock and SM at the sampled clock)
+    flops = 4.0 * B * Hq * g * cfg.kv_len * D
+    peaks = json.load(open(peaks_path)) if os.path.exists(peaks_path) else {}
+    bf16_peak = float(peaks.get("bf16_tflops_sustained", 1400.0))
+    exps = float(B * Hq * g * cfg.kv_len)
+    sm_mhz = clocks.summary().get("sm_mhz") or 1965.0
+    n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "peak_source": peak_src, "kernel": "verify attention (one layer)",
                 "us_per_launch": us_per_launch, "bytes_per_launch": bytes_per_launch,
-                "frac_of_nominal_8000": achieved / 8000.0}
+                "us_per_launch_median": attn_ms[len(attn_ms) // 2] * 1e3 / cfg.layers,
+                "us_per_launch_min": attn_ms[0] * 1e3 / cfg.layers,
+                "frac_of_nominal_8000": achieved / 8000.0,
+                "tensor_tflops": flops / (us_per_launch * 1e-6) / 1e12,
+                "tensor_frac_of_measured_bf16": flops / (us_per_launch * 1e-6) / 1e12 / bf16_peak,
+                "mufu_frac": exps / (us_per_launch * 1e-6) / (16.0 * n_sm * sm_mhz * 1e6)}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
