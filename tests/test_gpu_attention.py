@@ -86,6 +86,17 @@ def test_split_count_invariance_and_reproducibility(ctx, oracle_mod, kernel):
 
 
 @pytest.mark.parametrize("kernel", KERNELS)
+def test_more_splits_than_one_combine_batch(ctx, oracle_mod, kernel):
+    """The combine merges 32 splits per round trip: 45 splits take two rounds, the second
+    with a moved reference exponent (the scores rise along the cache)."""
+    case = _case(14, 1, 6, 8, 2, 128, 6016, [6000], [[100, 5000]])
+    q, k, v, kv_len, span = case
+    ramp = np.linspace(0.0, 3.0, k.shape[2], dtype=np.float32)[None, None, :, None]
+    k = W.f32_to_bf16_bits(W.bf16_bits_to_f32(k) + ramp * np.sign(W.bf16_bits_to_f32(q).mean()))
+    _check(ctx, oracle_mod, (q, k, v, kv_len, span), n_split=45, kernel=kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
 def test_peaked_scores(ctx, oracle_mod, kernel):
     """Scores with a wide dynamic range that rise along the cache, so the
     running maximum moves repeatedly and late keys dominate."""
