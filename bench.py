@@ -49,6 +49,11 @@ def parse():
     ap.add_argument("--sweep", action="store_true",
                     help="run the head-shape sweep (BASELINE config 4): gamma x KV length x batch, one layer "
                          "per point; the JSON line then carries the per-point table under \"sweep\"")
+    ap.add_argument("--lam", type=float, default=None,
+                    help="loosening ratio lambda of the rule (the config's 0.7 by default; the paper's "
+                         "sensitivity table runs 0.0, 0.2, 0.5, 0.7, 0.9)")
+    ap.add_argument("--top-n", type=int, default=10,
+                    help="N of the cosine Top-N relevance score timed beside the step (the paper runs 1, 10, 100)")
     ap.add_argument("--layers", type=int, default=0,
                     help="override the config's layer count (a smaller case of the same kernel for "
                          "profiler captures; the line then says so and is not a bench value)")
@@ -427,7 +432,7 @@ def run_ours(args, cfg):
             "cuda_graph": graph_attn is not None, "roofline": roofline, "clocks": clocks.summary()}
 
     if not args.no_next_rows and world == 1:
-        line["next_rows"] = {"visual_relevance": time_visual_relevance(cfg, ctx, stream, torch, dev, peak),
+        line["next_rows"] = {"visual_relevance": time_visual_relevance(cfg, ctx, stream, torch, dev, peak, args.top_n),
                              "paged_attention": time_paged_attention(cfg, ctx, stream, ks, vs_, qs, torch, dev, peak)}
 
     # end to end through the host-buffer entry points
@@ -445,7 +450,7 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
-def time_visual_relevance(cfg, ctx, stream, torch, dev, peak):
+def time_visual_relevance(cfg, ctx, stream, torch, dev, peak, top_n=10):
     """The paper's own relevance score (Eq. 4) on the config's visual span and
     hidden size, N = 10: not part of the verify step this benchmark times (the
     step scores positions by the attention's visual mass), measured beside it.
@@ -462,7 +467,7 @@ def time_visual_relevance(cfg, ctx, stream, torch, dev, peak):
         for c in range(2):
             ctx.row_inv_norms(B * lv, d, hv[c], inv[c])
         for c in range(2):
-            ctx.visual_relevance(B, g, lv, d, hd, hv[c], inv[c], 10, rel)
+            ctx.visual_relevance(B, g, lv, d, hd, hv[c], inv[c], top_n, rel)
     stream.synchronize()
     reps = 10
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -470,13 +475,13 @@ def time_visual_relevance(cfg, ctx, stream, torch, dev, peak):
         e0.record(stream)
         for _ in range(reps):
             for c in range(2):
-                ctx.visual_relevance(B, g, lv, d, hd, hv[c], inv[c], 10, rel)
+                ctx.visual_relevance(B, g, lv, d, hd, hv[c], inv[c], top_n, rel)
         e1.record(stream)
     stream.synchronize()
     us = e0.elapsed_time(e1) * 1e3 / (2 * reps)
     nbytes = B * lv * d * 2 + B * lv * 4
     gbs = nbytes / (us * 1e-6) / 1e9
-    return {"us_per_call": us, "n_visual": lv, "dim": d, "top_n": 10, "bytes_per_call": nbytes,
+    return {"us_per_call": us, "n_visual": lv, "dim": d, "top_n": top_n, "bytes_per_call": nbytes,
             "achieved_gbs": gbs, "frac_of_peak": gbs / peak, "launches_per_call": 3}
 
 
@@ -696,6 +701,8 @@ def main():
     cfg = W.CONFIGS[args.config]
     if args.layers > 0:
         cfg = dataclasses.replace(cfg, layers=args.layers)
+    if args.lam is not None:
+        cfg = dataclasses.replace(cfg, lam=args.lam)
     if args.impl == "reference":
         run_reference(args, cfg)
     else:
