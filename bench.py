@@ -433,7 +433,8 @@ def run_ours(args, cfg):
 
     if not args.no_next_rows and world == 1:
         line["next_rows"] = {"visual_relevance": time_visual_relevance(cfg, ctx, stream, torch, dev, peak, args.top_n),
-                             "paged_attention": time_paged_attention(cfg, ctx, stream, ks, vs_, qs, torch, dev, peak)}
+                             "paged_attention": time_paged_attention(cfg, ctx, stream, ks, vs_, qs, torch, dev, peak),
+                             "several_spans": time_span_layer(cfg, ctx, stream, ks, vs_, qs, torch, dev)}
 
     # end to end through the host-buffer entry points
     if not args.no_e2e:
@@ -483,6 +484,50 @@ def time_visual_relevance(cfg, ctx, stream, torch, dev, peak, top_n=10):
     gbs = nbytes / (us * 1e-6) / 1e9
     return {"us_per_call": us, "n_visual": lv, "dim": d, "top_n": top_n, "bytes_per_call": nbytes,
             "achieved_gbs": gbs, "frac_of_peak": gbs / peak, "launches_per_call": 3}
+
+
+def time_span_layer(cfg, ctx, stream, ks, vs_, qs, torch, dev):
+    """The last layer's attention with the visual span cut into frames of 196 positions
+    with 3 positions of text between them (only the layer whose mass feeds the rule needs
+    the union of the spans): time of that one call against the plain call on the hull."""
+    from paper_2604_05650_b200 import binding
+    B, g, Hq, Hkv, D, L = cfg.batch, cfg.gamma, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.kv_len
+    frames, pos = [], cfg.span[0]
+    while pos + 196 <= cfg.span[1] and len(frames) < 200:
+        frames.append([pos, pos + 196])
+        pos += 199
+    spans = np.tile(np.asarray([frames], dtype=np.int32), (B, 1, 1))
+    hull = np.tile(np.asarray([[frames[0][0], frames[-1][1]]], dtype=np.int32), (B, 1))
+    out = torch.empty((B, g, Hq, D), dtype=torch.bfloat16, device=dev)
+    mass = torch.empty((B, g, Hq), dtype=torch.float32, device=dev)
+    shape = binding.attn_shape(B, g, Hq, Hkv, D, L, 0, 0)
+    kv_len = np.full((B,), L, dtype=np.int32)
+    n = min(4, len(ks))
+
+    def timed(call):
+        with torch.cuda.stream(stream):
+            for l in range(n):
+                call(l)
+            stream.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                ctx.set_stream(torch.cuda.current_stream().cuda_stream)
+                for l in range(n):
+                    call(l)
+            ctx.set_stream(stream.cuda_stream)
+            graph.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(5):
+                graph.replay()
+            e1.record(stream)
+        stream.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (5 * n)
+
+    us_spans = timed(lambda l: ctx.verify_attention_spans(shape, qs[l], ks[l], vs_[l], kv_len, spans, out, mass))
+    us_hull = timed(lambda l: ctx.verify_attention(shape, qs[l], ks[l], vs_[l], kv_len, hull, out, mass))
+    return {"n_spans": len(frames), "gap_positions": 3 * (len(frames) - 1), "us_per_call": us_spans,
+            "us_per_call_one_span": us_hull, "note": "graph replays of four layers' calls"}
 
 
 def time_paged_attention(cfg, ctx, stream, ks, vs_, qs, torch, dev, peak):

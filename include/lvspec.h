@@ -197,6 +197,28 @@ lvspec_status_t lvspec_verify_attention_tree(lvspec_ctx_t *ctx, const lvspec_att
 lvspec_status_t lvspec_select_branch(lvspec_ctx_t *ctx, int32_t batch, int32_t n_branches,
                                      const int32_t *accept_len, int32_t *best_branch, int32_t *best_len);
 
+/* lvspec_verify_attention with SEVERAL visual spans per sequence (a video whose
+ * frames are separated by text: time stamps, captions).  The paper scores a draft
+ * token against the visual tokens as a set (Eq. 4); on this path the score is the
+ * attention mass on them, so the set is the union of the spans:
+ *
+ *   visual_mass[b,g,h] = sum of p_j over j in the union of the spans, j < visible
+ *
+ *   visual_spans  host, int32 [B][n_spans][2]: [start, end) each, sorted and
+ *                 disjoint within a sequence, inside 0..kv_len[b]-gamma; an empty
+ *                 span (start == end) is padding.  At most 241 spans per sequence.
+ *
+ * `out` and all else are as for lvspec_verify_attention.  The attention kernels run
+ * on the hull of the spans; one more small kernel per sequence then takes off the
+ * mass of the positions between them (these are few), which it recomputes in fp32
+ * from q, k and the softmax denominators.  n_split = 1 is UNSUPPORTED with
+ * LVSPEC_KERNEL_TCGEN05 (the denominators come from the merge of the splits; the
+ * automatic choice takes care of it). */
+lvspec_status_t lvspec_verify_attention_spans(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                              const void *q, const void *k_cache, const void *v_cache,
+                                              const int32_t *kv_len, int32_t n_spans,
+                                              const int32_t *visual_spans, void *out, float *visual_mass);
+
 /* lvspec_verify_attention on a PAGED cache (a serving engine's layout; the paper's
  * runs keep one contiguous cache per sequence, Sec. "Experimental Setup", so this is a
  * layout variant of Eq. 1, not another operation).  K and V live in pools of

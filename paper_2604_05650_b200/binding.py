@@ -31,6 +31,7 @@ EXPORTS = (
     "lvspec_loose_accept_static", "lvspec_row_inv_norms", "lvspec_visual_relevance",
     "lvspec_selftest_wait_expiry", "lvspec_loose_accept_emit",
     "lvspec_verify_attention_tree", "lvspec_select_branch", "lvspec_verify_attention_paged",
+    "lvspec_verify_attention_spans",
 )
 
 
@@ -88,6 +89,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lvspec_verify_attention_tree.argtypes = [vp, S, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.lvspec_select_branch.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.lvspec_verify_attention_paged.argtypes = [vp, S, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.lvspec_verify_attention_spans.argtypes = [vp, S, vp, vp, vp, vp, i32, vp, vp, vp]
     lib.lvspec_loose_accept_emit.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp, vp, vp, vp, vp]
     lib.lvspec_row_inv_norms.argtypes = [vp, ctypes.c_int64, i32, vp, vp]
     lib.lvspec_visual_relevance.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, i32, vp]
@@ -200,6 +202,17 @@ class Context:
             self._h, ctypes.byref(shape), int(page_size), int(n_pages), _addr(q), _addr(k_pool),
             _addr(v_pool), _addr(block_table), kv_len.ctypes.data, span.ctypes.data, _addr(out),
             _addr(visual_mass)))
+
+    def verify_attention_spans(self, shape: AttnShape, q, k_cache, v_cache, kv_len, visual_spans,
+                               out, visual_mass) -> None:
+        """visual_spans: host int32 [B, n_spans, 2], sorted and disjoint per sequence."""
+        kv_len = _i32(kv_len)
+        spans = np.ascontiguousarray(np.asarray(visual_spans, dtype=np.int32))
+        if spans.ndim != 3 or spans.shape[0] != shape.batch or spans.shape[2] != 2 or kv_len.size != shape.batch:
+            raise ValueError("visual_spans needs shape [B, n_spans, 2] and kv_len B entries")
+        self._check(self._lib.lvspec_verify_attention_spans(
+            self._h, ctypes.byref(shape), _addr(q), _addr(k_cache), _addr(v_cache), kv_len.ctypes.data,
+            int(spans.shape[1]), spans.ctypes.data, _addr(out), _addr(visual_mass)))
 
     def select_branch(self, batch, n_branches, accept_len, best_branch, best_len) -> None:
         self._check(self._lib.lvspec_select_branch(self._h, int(batch), int(n_branches), _addr(accept_len),

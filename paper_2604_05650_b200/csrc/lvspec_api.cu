@@ -7,6 +7,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <vector>
 
 #include "lvspec_internal.h"
 
@@ -155,7 +156,8 @@ struct PagedCache {          // page pools instead of one contiguous cache per s
 
 lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, const SeqInfo &seq,
                               int max_len, const void *q, const void *k, const void *v, void *out,
-                              float *mass, int branch_len = 0, const PagedCache *paged = nullptr)
+                              float *mass, int branch_len = 0, const PagedCache *paged = nullptr,
+                              float **lse2 = nullptr)
 {
     AttnParams p;
     std::memset(&p, 0, sizeof p);
@@ -186,10 +188,15 @@ lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, con
 
     const size_t o_bytes = part_o_elems(p) * sizeof(float);
     const size_t st_bytes = part_stat_elems(p) * sizeof(float);
-    lvspec_status_t st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, o_bytes + st_bytes, false);
+    const size_t lse_bytes = lse2 ? (size_t)p.B * p.gamma * p.Hq * sizeof(float) : 0;
+    lvspec_status_t st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, o_bytes + st_bytes + lse_bytes, false);
     if (st != LVSPEC_OK) return st;
     p.part_o = static_cast<float *>(ctx->scratch);
     p.part_stat = reinterpret_cast<float *>(static_cast<char *>(ctx->scratch) + o_bytes);
+    if (lse2) {
+        p.lse2 = reinterpret_cast<float *>(static_cast<char *>(ctx->scratch) + o_bytes + st_bytes);
+        *lse2 = p.lse2;
+    }
 
     int launches = 0;
     cudaError_t e;
@@ -446,6 +453,90 @@ lvspec_status_t lvspec_verify_attention_tree(lvspec_ctx_t *ctx, const lvspec_att
     if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
     return run_attention(ctx, shape, seq, max_len, q, k_cache, v_cache, out, visual_mass,
                          shape->gamma / n_branches);
+}
+
+lvspec_status_t lvspec_verify_attention_spans(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                              const void *q, const void *k_cache, const void *v_cache,
+                                              const int32_t *kv_len, int32_t n_spans,
+                                              const int32_t *visual_spans, void *out, float *visual_mass)
+{
+    if (!ctx) return LVSPEC_ERR_INVALID_ARG;
+    if (!shape || !visual_spans || !kv_len) return fail(ctx, LVSPEC_ERR_INVALID_ARG, "null argument");
+    if (n_spans < 1 || n_spans > kMaxGaps + 1)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "n_spans outside 1.." + std::to_string(kMaxGaps + 1));
+    if (shape->batch < 1 || shape->batch > LVSPEC_MAX_BATCH)
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "batch outside 1..LVSPEC_MAX_BATCH");
+    // per sequence: the hull of the non-empty spans, and the ranges between them
+    std::vector<int32_t> hull(2 * (size_t)shape->batch);
+    std::vector<std::vector<int32_t>> gaps(shape->batch);
+    for (int b = 0; b < shape->batch; ++b) {
+        int first = -1, last_end = 0;
+        for (int i = 0; i < n_spans; ++i) {
+            const int s = visual_spans[((size_t)b * n_spans + i) * 2], e = visual_spans[((size_t)b * n_spans + i) * 2 + 1];
+            if (s < 0 || e < s || e > kv_len[b] - shape->gamma)
+                return fail(ctx, LVSPEC_ERR_INVALID_ARG, "a visual span lies outside 0..kv_len-gamma");
+            if (s == e) continue;                      // padding
+            if (first < 0) first = s;
+            else {
+                if (s < last_end)
+                    return fail(ctx, LVSPEC_ERR_INVALID_ARG, "visual spans must be sorted and disjoint");
+                if (s > last_end) { gaps[b].push_back(last_end); gaps[b].push_back(s); }
+            }
+            last_end = e;
+        }
+        hull[2 * b] = first < 0 ? 0 : first;
+        hull[2 * b + 1] = first < 0 ? 0 : last_end;
+    }
+    SeqInfo seq;
+    int max_len = 0;
+    lvspec_status_t st = check_attention(ctx, shape, q, k_cache, v_cache, kv_len, hull.data(), out,
+                                         visual_mass, true, &seq, &max_len);
+    if (st != LVSPEC_OK) return st;
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
+    // the log2 denominators come from the combine kernel: at least two splits where the
+    // tensor-core kernel would otherwise finish alone (the plain kernel always combines)
+    lvspec_attn_shape_t s = *shape;
+    if (resolve_kernel(&s) == LVSPEC_KERNEL_TCGEN05 && s.n_split == 0 && choose_splits(ctx, &s, max_len) < 2) {
+        if (max_len > 128) s.n_split = 2;
+        else s.kernel = LVSPEC_KERNEL_SIMT;
+    }
+    if (resolve_kernel(&s) == LVSPEC_KERNEL_TCGEN05 && s.n_split == 1)
+        return fail(ctx, LVSPEC_ERR_UNSUPPORTED, "several spans need n_split != 1 with the tcgen05 kernel");
+    float *lse2 = nullptr;
+    st = run_attention(ctx, &s, seq, max_len, q, k_cache, v_cache, out, visual_mass, 0, nullptr, &lse2);
+    if (st != LVSPEC_OK) return st;
+    for (int b = 0; b < shape->batch; ++b) {
+        if (gaps[b].empty()) continue;
+        GapParams g;
+        std::memset(&g, 0, sizeof g);
+        g.q = static_cast<const uint16_t *>(q);
+        g.k = static_cast<const uint16_t *>(k_cache);
+        g.lse2 = lse2;
+        g.mass = visual_mass;
+        g.b = b;
+        g.gamma = shape->gamma;
+        g.Hq = shape->n_q_heads;
+        g.Hkv = shape->n_kv_heads;
+        g.D = shape->head_dim;
+        g.Lmax = shape->kv_capacity;
+        g.G = g.Hq / g.Hkv;
+        g.M = g.gamma * g.G;
+        g.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)g.D));
+        g.n_gaps = (int)gaps[b].size() / 2;
+        int flat = 0;
+        for (int i = 0; i < g.n_gaps; ++i) {
+            g.gap_start[i] = gaps[b][2 * i];
+            g.gap_first[i] = flat;
+            flat += gaps[b][2 * i + 1] - gaps[b][2 * i];
+        }
+        g.gap_first[g.n_gaps] = flat;
+        int launches = 0;
+        e = launch_gap_mass(g, ctx->stream, &launches);
+        ctx->launches += launches;
+        if (e != cudaSuccess) return cuda_fail(ctx, "gap mass kernel launch", e);
+    }
+    return LVSPEC_OK;
 }
 
 lvspec_status_t lvspec_verify_attention_paged(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,

@@ -23,6 +23,7 @@ struct AttnParams {
     float *mass;           // [B, gamma, Hq]
     float *part_o;         // [B, Hkv, n_split, M, D] fp32, unnormalised
     float *part_stat;      // [B, Hkv, n_split, M, 4]: m (log2 units), l, l_vis, unused
+    float *lse2;           // optional [B, gamma, Hq]: log2 of the softmax denominator, written by the combine
     uint32_t *status;      // device status word
     int32_t B, gamma, Hq, Hkv, D, Lmax, G, M, n_split;
     int32_t pdl;           // launch programmatically dependent on the previous kernel
@@ -59,6 +60,22 @@ bool attn_tc_supported(const AttnParams &p);
 cudaError_t launch_attn_tc(const AttnParams &p, const SeqInfo &seq, cudaStream_t stream,
                            int *launches);
 cudaError_t launch_attn_combine(const AttnParams &p, cudaStream_t stream, int *launches);
+
+// Several visual spans: the attention runs on their hull, then the probability mass of
+// the positions between the spans (at most kMaxGaps ranges per sequence) is taken off.
+constexpr int kMaxGaps = 240;
+struct GapParams {
+    const uint16_t *q;     // [B, gamma, Hq, D]
+    const uint16_t *k;     // [B, Hkv, Lmax, D]
+    const float *lse2;     // [B, gamma, Hq]
+    float *mass;           // [B, gamma, Hq], corrected in place
+    int32_t b, gamma, Hq, Hkv, D, Lmax, G, M;
+    float scale_log2;
+    int32_t n_gaps;
+    int32_t gap_start[kMaxGaps];        // first cache position of each gap
+    int32_t gap_first[kMaxGaps + 1];    // gaps laid end to end: index of each gap's first position; [n_gaps] = total
+};
+cudaError_t launch_gap_mass(const GapParams &p, cudaStream_t stream, int *launches);
 
 struct AcceptParams {
     const float *logits;      // [B, gamma, V]

@@ -237,6 +237,7 @@ __global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const 
     const size_t row = ((size_t)b * p.gamma + g) * p.Hq + kvh * p.G + hg;
     uint16_t *out_row = p.out + row * D + lane * 4;
     float *mass_row = p.mass + row;
+    float *lse_row = p.lse2 ? p.lse2 + row : nullptr;
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     float m_run = -INFINITY, l = 0.f, lv = 0.f;
@@ -296,7 +297,10 @@ __global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const 
         pk.y = *reinterpret_cast<uint32_t *>(&hi);
         *reinterpret_cast<uint2 *>(out_row) = pk;
     }
-    if (lane == 0) *mass_row = lv * inv;
+    if (lane == 0) {
+        *mass_row = lv * inv;
+        if (lse_row) *lse_row = m_run + log2f(l);
+    }
 }
 
 }  // namespace
