@@ -14,6 +14,11 @@
  *       vocabulary-wide argmax per draft position, then the rule of Sec. 3.2
  *       and 3.3 (Eq. 5-7) and the accepted length of Eq. 2.
  *
+ * Around them, each documented at its declaration: the attention on a paged
+ * cache, with several visual spans, and on a draft-token tree; the acceptance
+ * pass with the emit step, with host buffers, and without any allocation; the
+ * paper's own relevance score (Eq. 4) as an alternative input to the rule.
+ *
  * Conventions
  *   - "device" pointers are CUDA global memory of the context's device; "host"
  *     pointers are ordinary host memory.  The caller owns every buffer it
@@ -22,7 +27,8 @@
  *     shapes given at each call; device tensors must be 16-byte aligned.
  *   - Device calls enqueue work on the context's stream and return without
  *     synchronising.  The return value reports argument and launch errors only.
- *     A call that returns anything but LVSPEC_OK has launched nothing.
+ *     A call refused for its arguments (INVALID_ARG, UNSUPPORTED) has launched
+ *     nothing.
  *   - A context owns scratch memory on its device and is not thread-safe.
  *     Calls on one context must not overlap on the GPU with each other unless
  *     they are ordered on the same stream.
