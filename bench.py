@@ -39,7 +39,7 @@ def parse():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=2, help="BASELINE config id (1, 2 or 3)")
+    ap.add_argument("--config", type=int, default=2, help="workload config id (1, 2 or 3)")
     ap.add_argument("--kernel", type=int, default=0, help="attention kernel selector (0 = default)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -47,7 +47,7 @@ def parse():
     ap.add_argument("--no-next-rows", action="store_true",
                     help="skip the timing of the paper's own relevance score (not part of the step)")
     ap.add_argument("--sweep", action="store_true",
-                    help="run the head-shape sweep (BASELINE config 4): gamma x KV length x batch, one layer "
+                    help="run the head-shape sweep (workload config 4): gamma x KV length x batch, one layer "
                          "per point; the JSON line then carries the per-point table under \"sweep\"")
     ap.add_argument("--lam", type=float, default=None,
                     help="loosening ratio lambda of the rule (the config's 0.7 by default; the paper's "
@@ -212,7 +212,7 @@ def run_reference(args, cfg):
 
 
 def workload_desc(cfg, n_gpus):
-    return {"workload": f"BASELINE config {cfg_id_of(cfg)}: {cfg.name}-shaped verify step, {cfg.layers} layers, "
+    return {"workload": f"workload config {cfg_id_of(cfg)}: {cfg.name}-shaped verify step, {cfg.layers} layers, "
                         f"batch {cfg.batch}, gamma {cfg.gamma}, heads {cfg.n_q_heads}/{cfg.n_kv_heads}x{cfg.head_dim}, "
                         f"KV {cfg.kv_len} ({cfg.span[1] - cfg.span[0]} visual), vocab {cfg.vocab}",
             "kv_bytes_per_step": cfg.kv_bytes_per_layer * cfg.layers,
@@ -635,7 +635,7 @@ def run_e2e(args, cfg, ctx, stream, qs, ks, vs_, logits, draft, torch, dev, worl
 
 
 def run_sweep(args):
-    """BASELINE config 4: the 40/8x128 head shape, one layer, gamma x KV length x
+    """workload config 4: the 40/8x128 head shape, one layer, gamma x KV length x
     batch.  Per point: time of one attention call and of the acceptance pass,
     achieved HBM GB/s of the attention call against the measured peak, verified
     tokens/s of the single-layer step.  Each point rotates over enough distinct
@@ -730,7 +730,7 @@ def run_sweep(args):
     line = {"metric": METRIC, "value": tok_total / (ms_total * 1e-3), "unit": UNIT, "n_gpus": 1,
             "steps": len(points), "warmup": 3, "ms_per_step": ms_total / len(points), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "BASELINE config 4: sweep on the 40/8x128 head shape, one layer per point, "
+            "config": {"workload": "workload config 4: sweep on the 40/8x128 head shape, one layer per point, "
                                    "gamma {4,8,16} x KV {4K,16K,64K,128K} x batch {1,4,16}, 75% visual",
                        "l2": "each point rotates over >= 256 MB of distinct K/V buffers"},
             "device_status": status, "clocks": clocks.summary(), "peak_hbm_gbs": peak, "sweep": points}
