@@ -67,9 +67,19 @@ def test_config0(ctx, oracle_mod, kernel):
     (1, 1, 4, 4, 64, 300, [257], [[3, 200]], 2),               # gamma 1, G 1
     (2, 4, 28, 4, 128, 600, [600, 599], [[256, 500], [1, 2]], 0),   # G = 7 (M = 28)
     (1, 8, 16, 1, 64, 130, [130], [[20, 100]], 64),            # more splits than tiles
+    (1, 16, 16, 2, 128, 1500, [1500], [[100, 1200]], 4),       # M = 128: the most rows a KV head takes
+    (1, 64, 4, 2, 128, 900, [900], [[0, 700]], 1),             # gamma 64 (the most), one split
+    (2, 5, 10, 2, 128, 640, [640, 517], [[7, 300], [0, 512]], 3),   # M = 25: last chunk of 8 columns not full
+    (1, 13, 26, 2, 128, 1300, [1290], [[200, 1000]], 0),       # M = 169 > 128 rows: refused
 ])
 def test_small_shapes(ctx, oracle_mod, shape, kernel):
     B, gamma, Hq, Hkv, D, Lmax, kv_len, span, n_split = shape
+    if gamma * (Hq // Hkv) > 128:
+        from paper_2604_05650_b200 import binding
+        with pytest.raises(binding.LvspecError) as e:
+            _check(ctx, oracle_mod, _case(11, B, gamma, Hq, Hkv, D, Lmax, kv_len, span), kernel=kernel)
+        assert e.value.status == binding.ERR_UNSUPPORTED
+        return
     _check(ctx, oracle_mod, _case(11, B, gamma, Hq, Hkv, D, Lmax, kv_len, span),
            n_split=n_split, kernel=kernel)
 
