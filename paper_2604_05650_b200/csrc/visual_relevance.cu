@@ -62,6 +62,10 @@ __global__ void __launch_bounds__(kPrepThreads)
 draft_prep_kernel(const uint16_t *hd, int B, int K, int NP, int dim, uint16_t *hd_pad, float *dinv)
 {
     __shared__ float part[kPrepThreads / 32];
+    // the streaming kernel may be scheduled at once (it sets itself up, then waits for
+    // this grid); this grid waits for whatever ran before it in the stream
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int r = blockIdx.x;                       // padded row index over B * NP
     const int b = r / NP, k = r - b * NP;
     uint4 *dst = reinterpret_cast<uint4 *>(hd_pad + (size_t)r * dim);
@@ -578,10 +582,17 @@ cudaError_t launch_visual_relevance(const RelevanceParams &p, cudaStream_t strea
     o = (o + 1023) & ~size_t(1023);
     float *dinv = reinterpret_cast<float *>(reinterpret_cast<char *>(p.cos_t) + o);
 
-    draft_prep_kernel<<<p.B * NP, kPrepThreads, 0, stream>>>(
-        p.h_draft, p.B, p.K, NP, p.d, hd_pad, dinv);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg0 = {};
+    cfg0.gridDim = dim3((unsigned)(p.B * NP), 1, 1);
+    cfg0.blockDim = dim3(kPrepThreads, 1, 1);
+    cfg0.stream = stream;
+    cfg0.attrs = attr;
+    cfg0.numAttrs = 1;
+    cudaError_t err = cudaLaunchKernelEx(&cfg0, draft_prep_kernel, p.h_draft, p.B, p.K, NP, p.d, hd_pad, dinv);
     ++*launches;
-    cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
 
     CosParams P;
@@ -616,9 +627,6 @@ cudaError_t launch_visual_relevance(const RelevanceParams &p, cudaStream_t strea
     const size_t smem = (size_t)P.smem_bytes + 1024;
     err = cudaFuncSetAttribute(cos_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)n_cta, 1, 1);
     cfg.blockDim = dim3(kCosThreads, 1, 1);
