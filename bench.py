@@ -629,9 +629,47 @@ def run_e2e(args, cfg, ctx, stream, qs, ks, vs_, logits, draft, torch, dev, worl
     h2d = cfg.layers * (hq[0].numel() * 2 + 2 * hk[0].numel() * 2) + hlog.numel() * 4 + hdraft.numel() * 4 \
         + hmass.numel() * 4
     d2h = cfg.layers * (hout.numel() * 2 + hmass.numel() * 4) + hlen.numel() * 4
+    # The same step as a serving loop sees it: the caches are state and stay on the device;
+    # what crosses PCIe every step is what the step is given (the draft queries of every
+    # layer, the target logits, the draft tokens) and what it returns (the accepted length).
+    dq = [torch.empty_like(t) for t in qs]
+    dlog, ddraft = torch.empty_like(logits), torch.empty_like(draft)
+    dout = torch.empty((B, g, Hq, D), dtype=torch.bfloat16, device=dev)
+    dmass = torch.empty((B, g, Hq), dtype=torch.float32, device=dev)
+    dlen = torch.zeros((B,), dtype=torch.int32, device=dev)
+
+    def resident_step():
+        with torch.cuda.stream(stream):
+            for l in range(cfg.layers):
+                dq[l].copy_(hq[l], non_blocking=True)
+            dlog.copy_(hlog, non_blocking=True)
+            ddraft.copy_(hdraft, non_blocking=True)
+            for l in range(cfg.layers):
+                ctx.verify_attention(shape, dq[l], ks[l], vs_[l], kv_len, span, dout, dmass)
+            ctx.loose_accept(B, g, cfg.vocab, Hq, dlog, ddraft, dmass, dlen, cfg.shift_window, lam=cfg.lam)
+            hlen.copy_(dlen, non_blocking=True)
+        stream.synchronize()
+
+    resident_step()
+    barrier()
+    r_steps = max(3, min(args.steps, 20))
+    torch.cuda.synchronize(dev)
+    ev0.record(stream)
+    for _ in range(r_steps):
+        resident_step()
+    ev1.record(stream)
+    stream.synchronize()
+    barrier()
+    ms_res = slowest_rank_ms(ev0.elapsed_time(ev1) / r_steps, world, dist, dev)
+    res_h2d = cfg.layers * hq[0].numel() * 2 + hlog.numel() * 4 + hdraft.numel() * 4
     return {"value": whole_job_tokens_per_s(world, B, g, ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": ms, "steps": steps,
-            "note": "K/V caches of every layer cross PCIe each step"}
+            "note": "K/V caches of every layer cross PCIe each step",
+            "kv_resident": {"value": whole_job_tokens_per_s(world, B, g, ms_res), "unit": UNIT,
+                            "h2d_bytes_per_step": res_h2d, "d2h_bytes_per_step": hlen.numel() * 4,
+                            "ms_per_step": ms_res, "steps": r_steps,
+                            "note": "caches resident on the device; queries, logits and drafts from pinned host "
+                                    "memory, accepted length back, a host synchronisation every step, plain launches"}}
 
 
 def run_sweep(args):
