@@ -632,21 +632,39 @@ def run_e2e(args, cfg, ctx, stream, qs, ks, vs_, logits, draft, torch, dev, worl
     # The same step as a serving loop sees it: the caches are state and stay on the device;
     # what crosses PCIe every step is what the step is given (the draft queries of every
     # layer, the target logits, the draft tokens) and what it returns (the accepted length).
-    dq = [torch.empty_like(t) for t in qs]
+    hq_all = torch.stack([t for t in hq]).pin_memory()          # one copy per step for all layers' queries
+    dq_all = torch.empty(hq_all.shape, dtype=hq_all.dtype, device=dev)
+    dq = [dq_all[l] for l in range(cfg.layers)]
     dlog, ddraft = torch.empty_like(logits), torch.empty_like(draft)
     dout = torch.empty((B, g, Hq, D), dtype=torch.bfloat16, device=dev)
     dmass = torch.empty((B, g, Hq), dtype=torch.float32, device=dev)
     dlen = torch.zeros((B,), dtype=torch.int32, device=dev)
 
+    def device_part():
+        for l in range(cfg.layers):
+            ctx.verify_attention(shape, dq[l], ks[l], vs_[l], kv_len, span, dout, dmass)
+        ctx.loose_accept(B, g, cfg.vocab, Hq, dlog, ddraft, dmass, dlen, cfg.shift_window, lam=cfg.lam)
+
+    step_graph = None
+    if not args.no_graph:
+        with torch.cuda.stream(stream):
+            device_part()
+            stream.synchronize()
+            step_graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(step_graph, stream=stream):
+                ctx.set_stream(torch.cuda.current_stream().cuda_stream)
+                device_part()
+            ctx.set_stream(stream.cuda_stream)
+
     def resident_step():
         with torch.cuda.stream(stream):
-            for l in range(cfg.layers):
-                dq[l].copy_(hq[l], non_blocking=True)
+            dq_all.copy_(hq_all, non_blocking=True)
             dlog.copy_(hlog, non_blocking=True)
             ddraft.copy_(hdraft, non_blocking=True)
-            for l in range(cfg.layers):
-                ctx.verify_attention(shape, dq[l], ks[l], vs_[l], kv_len, span, dout, dmass)
-            ctx.loose_accept(B, g, cfg.vocab, Hq, dlog, ddraft, dmass, dlen, cfg.shift_window, lam=cfg.lam)
+            if step_graph is not None:
+                step_graph.replay()
+            else:
+                device_part()
             hlen.copy_(dlen, non_blocking=True)
         stream.synchronize()
 
@@ -669,7 +687,8 @@ def run_e2e(args, cfg, ctx, stream, qs, ks, vs_, logits, draft, torch, dev, worl
                             "h2d_bytes_per_step": res_h2d, "d2h_bytes_per_step": hlen.numel() * 4,
                             "ms_per_step": ms_res, "steps": r_steps,
                             "note": "caches resident on the device; queries, logits and drafts from pinned host "
-                                    "memory, accepted length back, a host synchronisation every step, plain launches"}}
+                                    "memory, accepted length back, a host synchronisation every step; the device part is "
+                                    "one CUDA graph unless --no-graph"}}
 
 
 def run_sweep(args):
