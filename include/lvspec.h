@@ -48,7 +48,8 @@ typedef enum {
     LVSPEC_OK = 0,
     LVSPEC_ERR_INVALID_ARG = 1,  /* null pointer, bad shape, span or length out of range */
     LVSPEC_ERR_UNSUPPORTED = 2,  /* a shape the kernels do not cover (see each call) */
-    LVSPEC_ERR_WORKSPACE = 3,    /* scratch memory could not be allocated */
+    LVSPEC_ERR_WORKSPACE = 3,    /* scratch memory could not be allocated, or would have to grow
+                                    during a stream capture (see lvspec_reserve) */
     LVSPEC_ERR_CUDA = 4,         /* a CUDA runtime call failed; see lvspec_last_error */
     LVSPEC_ERR_TIMEOUT = 5       /* a bounded device-side wait ran out */
 } lvspec_status_t;
@@ -113,6 +114,9 @@ lvspec_status_t lvspec_set_stream(lvspec_ctx_t *ctx, void *cuda_stream);
  * `flags` (host) receives the LVSPEC_DEV_* bits.  Returns LVSPEC_ERR_TIMEOUT if
  * LVSPEC_DEV_WAIT_EXPIRED is set, LVSPEC_ERR_CUDA if the sync failed. */
 lvspec_status_t lvspec_device_status(lvspec_ctx_t *ctx, uint32_t *flags);
+/* The same call under the name "last device status": what the kernels launched
+ * since the previous reading have reported. */
+lvspec_status_t lvspec_last_device_status(lvspec_ctx_t *ctx, uint32_t *flags);
 
 /* Text of the last error recorded on this context (never NULL; valid until the
  * next call on the context).  `ctx` may be NULL: then the text describes why
@@ -128,6 +132,37 @@ uint64_t lvspec_launch_count(const lvspec_ctx_t *ctx);
  * `max_kv_len` (what n_split = 0 resolves to); 0 on invalid input. */
 int32_t lvspec_attention_splits(const lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
                                 int32_t max_kv_len);
+
+/* Scratch memory.  A context owns one scratch buffer on its device (split
+ * partials of the attention, argmax partials of the acceptance pass, cosines of
+ * the relevance score; never results).  A call that needs more than the context
+ * holds grows it: that synchronises the context's stream, frees and allocates,
+ * and so must not happen inside a CUDA-graph stream capture.  A caller that
+ * captures its calls, or that wants every allocation done at start-up, sizes the
+ * buffer first:
+ *
+ *   lvspec_*_workspace_bytes  bytes of scratch the call of that shape needs
+ *       (attention: any of the lvspec_verify_attention* forms with `shape`, the
+ *       longest sequence `max_kv_len` and the split choice `shape->n_split`;
+ *       accept: any of the lvspec_loose_accept* forms that take a context;
+ *       relevance: lvspec_visual_relevance).  0 on invalid input.
+ *   lvspec_reserve            grows the buffer to at least `workspace_bytes`
+ *       (the largest of the figures above); never shrinks it.
+ *   lvspec_workspace_capacity bytes the context holds now.
+ *
+ * While the context's stream is being captured, a call that would have to grow
+ * the buffer returns LVSPEC_ERR_WORKSPACE instead, launches nothing and leaves
+ * the capture valid; lvspec_reserve does the same.  The *_host forms also own
+ * device staging memory for their copies; they synchronise anyway and are not
+ * meant for capture. */
+size_t lvspec_attention_workspace_bytes(const lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                        int32_t max_kv_len);
+size_t lvspec_accept_workspace_bytes(const lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,
+                                     int32_t vocab);
+size_t lvspec_relevance_workspace_bytes(const lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,
+                                        int32_t n_visual, int32_t dim);
+size_t lvspec_workspace_capacity(const lvspec_ctx_t *ctx);
+lvspec_status_t lvspec_reserve(lvspec_ctx_t *ctx, size_t workspace_bytes);
 
 /* Self-test of the bounded device-side waits.  Every barrier wait in the kernels
  * of this library has a time limit (about two seconds); a wait that runs out

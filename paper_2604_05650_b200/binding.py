@@ -31,7 +31,9 @@ EXPORTS = (
     "lvspec_loose_accept_static", "lvspec_row_inv_norms", "lvspec_visual_relevance",
     "lvspec_selftest_wait_expiry", "lvspec_loose_accept_emit",
     "lvspec_verify_attention_tree", "lvspec_select_branch", "lvspec_verify_attention_paged",
-    "lvspec_verify_attention_spans",
+    "lvspec_verify_attention_spans", "lvspec_last_device_status",
+    "lvspec_attention_workspace_bytes", "lvspec_accept_workspace_bytes",
+    "lvspec_relevance_workspace_bytes", "lvspec_workspace_capacity", "lvspec_reserve",
 )
 
 
@@ -72,6 +74,17 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lvspec_destroy.argtypes = [vp]
     lib.lvspec_set_stream.argtypes = [vp, vp]
     lib.lvspec_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.lvspec_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+    sz = ctypes.c_size_t
+    lib.lvspec_attention_workspace_bytes.argtypes = [vp, S, i32]
+    lib.lvspec_attention_workspace_bytes.restype = sz
+    lib.lvspec_accept_workspace_bytes.argtypes = [vp, i32, i32, i32]
+    lib.lvspec_accept_workspace_bytes.restype = sz
+    lib.lvspec_relevance_workspace_bytes.argtypes = [vp, i32, i32, i32, i32]
+    lib.lvspec_relevance_workspace_bytes.restype = sz
+    lib.lvspec_workspace_capacity.argtypes = [vp]
+    lib.lvspec_workspace_capacity.restype = sz
+    lib.lvspec_reserve.argtypes = [vp, sz]
     lib.lvspec_last_error.argtypes = [vp]
     lib.lvspec_last_error.restype = ctypes.c_char_p
     lib.lvspec_status_string.argtypes = [ctypes.c_int]
@@ -165,6 +178,23 @@ class Context:
 
     def selftest_wait_expiry(self, limit_ms: int = 5) -> None:
         self._check(self._lib.lvspec_selftest_wait_expiry(self._h, int(limit_ms)))
+
+    # -- scratch memory --------------------------------------------------------------
+    def attention_workspace_bytes(self, shape: AttnShape, max_kv_len: int) -> int:
+        return int(self._lib.lvspec_attention_workspace_bytes(self._h, ctypes.byref(shape), int(max_kv_len)))
+
+    def accept_workspace_bytes(self, batch, gamma, vocab) -> int:
+        return int(self._lib.lvspec_accept_workspace_bytes(self._h, int(batch), int(gamma), int(vocab)))
+
+    def relevance_workspace_bytes(self, batch, gamma, n_visual, dim) -> int:
+        return int(self._lib.lvspec_relevance_workspace_bytes(self._h, int(batch), int(gamma), int(n_visual),
+                                                              int(dim)))
+
+    def workspace_capacity(self) -> int:
+        return int(self._lib.lvspec_workspace_capacity(self._h))
+
+    def reserve(self, workspace_bytes: int) -> None:
+        self._check(self._lib.lvspec_reserve(self._h, int(workspace_bytes)))
 
     def launch_count(self) -> int:
         return int(self._lib.lvspec_launch_count(self._h))

@@ -47,9 +47,30 @@ lvspec_status_t cuda_fail(lvspec_ctx *ctx, const char *what, cudaError_t err)
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Is the context's stream being captured into a CUDA graph right now?  (On the legacy
+// default stream the query itself fails while another stream captures: that too counts.)
+bool stream_is_capturing(lvspec_ctx *ctx)
+{
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    const cudaError_t e = cudaStreamIsCapturing(ctx->stream, &cs);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return true;
+    }
+    return cs != cudaStreamCaptureStatusNone;
+}
+
+// Grows *buf to at least `want` bytes.  Growing synchronises the stream, frees and
+// allocates: none of that may happen while the stream is being captured, so there the
+// call is refused (the capture stays valid) and the caller is told to reserve first.
 lvspec_status_t ensure(lvspec_ctx *ctx, void **buf, size_t *have, size_t want, bool zero)
 {
     if (want <= *have) return LVSPEC_OK;
+    if (stream_is_capturing(ctx))
+        return fail(ctx, LVSPEC_ERR_WORKSPACE,
+                    "the call needs " + std::to_string(want) + " bytes of scratch memory, the context holds " +
+                        std::to_string(*have) + ", and memory cannot be grown while the stream is being "
+                        "captured: call lvspec_reserve (or run the call once) before the capture");
     if (*buf) {
         cudaError_t e = cudaStreamSynchronize(ctx->stream);
         if (e != cudaSuccess) return cuda_fail(ctx, "cudaStreamSynchronize", e);
@@ -98,6 +119,26 @@ int choose_splits(const lvspec_ctx *ctx, const lvspec_attn_shape_t *s, int max_k
     if (want > tiles) want = tiles;
     if (want > 256) want = 256;
     return want;
+}
+
+// Vocabulary slices of the acceptance kernel: enough CTAs for two per SM, at least 4096
+// elements each.
+int accept_vocab_slices(const lvspec_ctx *ctx, int rows, int vocab)
+{
+    int vs = (2 * ctx->n_sm + rows - 1) / rows;
+    const int max_vs = (vocab + 4095) / 4096;
+    if (vs > max_vs) vs = max_vs;
+    if (vs < 1) vs = 1;
+    return vs;
+}
+
+// Scratch bytes of one attention call: the split partials (fp32 rows and their
+// statistics) and, for the call with several spans, the log2 denominators.
+size_t attention_scratch_bytes(int B, int Hkv, int n_split, int M, int D, int gamma, int Hq, bool with_lse)
+{
+    const size_t units = (size_t)B * Hkv * n_split;
+    return units * M * D * sizeof(float) + units * M * 4 * sizeof(float) +
+           (with_lse ? (size_t)B * gamma * Hq * sizeof(float) : 0);
 }
 
 // Validation shared by the device and host forms.  On success fills seq.
@@ -188,8 +229,9 @@ lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, con
 
     const size_t o_bytes = part_o_elems(p) * sizeof(float);
     const size_t st_bytes = part_stat_elems(p) * sizeof(float);
-    const size_t lse_bytes = lse2 ? (size_t)p.B * p.gamma * p.Hq * sizeof(float) : 0;
-    lvspec_status_t st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, o_bytes + st_bytes + lse_bytes, false);
+    lvspec_status_t st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes,
+                                attention_scratch_bytes(p.B, p.Hkv, p.n_split, p.M, p.D, p.gamma, p.Hq,
+                                                        lse2 != nullptr), false);
     if (st != LVSPEC_OK) return st;
     p.part_o = static_cast<float *>(ctx->scratch);
     p.part_stat = reinterpret_cast<float *>(static_cast<char *>(ctx->scratch) + o_bytes);
@@ -277,12 +319,8 @@ lvspec_status_t run_accept(lvspec_ctx *ctx, int batch, int gamma, int vocab, int
     p.Hm = heads;
     p.n_loose = n_loose;
     p.window = window > gamma ? gamma : window;
-    // slices: enough CTAs for two per SM, at least 4096 elements each
-    int rows = batch * gamma;
-    int vs = (2 * ctx->n_sm + rows - 1) / rows;
-    const int max_vs = (vocab + 4095) / 4096;
-    if (vs > max_vs) vs = max_vs;
-    if (vs < 1) vs = 1;
+    const int rows = batch * gamma;
+    const int vs = accept_vocab_slices(ctx, rows, vocab);
     p.n_vsplit = vs;
     const size_t n_part = (size_t)rows * vs;
     lvspec_status_t st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes,
@@ -345,6 +383,8 @@ lvspec_status_t lvspec_create(lvspec_ctx_t **out, int device)
     if ((e = cudaMalloc(reinterpret_cast<void **>(&ctx->status), small)) != cudaSuccess ||
         (e = cudaMemset(ctx->status, 0, small)) != cudaSuccess) {
         g_create_error = std::string("status allocation: ") + cudaGetErrorString(e);
+        cudaFree(ctx->status);      // null when the allocation itself failed
+        cudaGetLastError();
         delete ctx;
         return LVSPEC_ERR_WORKSPACE;
     }
@@ -420,6 +460,49 @@ int32_t lvspec_attention_splits(const lvspec_ctx_t *ctx, const lvspec_attn_shape
 {
     if (!ctx || !shape || shape->batch < 1 || shape->n_kv_heads < 1 || max_kv_len < 1) return 0;
     return shape->n_split > 0 ? shape->n_split : choose_splits(ctx, shape, max_kv_len);
+}
+
+lvspec_status_t lvspec_last_device_status(lvspec_ctx_t *ctx, uint32_t *flags)
+{
+    return lvspec_device_status(ctx, flags);
+}
+
+size_t lvspec_attention_workspace_bytes(const lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                        int32_t max_kv_len)
+{
+    if (!ctx || !shape || shape->batch < 1 || shape->n_kv_heads < 1 || shape->gamma < 1 ||
+        shape->n_q_heads < shape->n_kv_heads || shape->head_dim < 1 || max_kv_len < 1 || shape->n_split < 0)
+        return 0;
+    const int n_split = shape->n_split > 0 ? shape->n_split : choose_splits(ctx, shape, max_kv_len);
+    // the call with several spans never runs the tensor-core kernel on a single split
+    const int n_eff = n_split < 2 ? 2 : n_split;
+    const int M = shape->gamma * (shape->n_q_heads / shape->n_kv_heads);
+    return attention_scratch_bytes(shape->batch, shape->n_kv_heads, n_eff, M, shape->head_dim, shape->gamma,
+                                   shape->n_q_heads, true);
+}
+
+size_t lvspec_accept_workspace_bytes(const lvspec_ctx_t *ctx, int32_t batch, int32_t gamma, int32_t vocab)
+{
+    if (!ctx || batch < 1 || gamma < 1 || vocab < 1) return 0;
+    const int rows = batch * gamma;
+    return (size_t)rows * accept_vocab_slices(ctx, rows, vocab) * (sizeof(float) + sizeof(int32_t));
+}
+
+size_t lvspec_relevance_workspace_bytes(const lvspec_ctx_t *ctx, int32_t batch, int32_t gamma,
+                                        int32_t n_visual, int32_t dim)
+{
+    if (!ctx || batch < 1 || gamma < 1 || n_visual < 1 || dim < 1) return 0;
+    return relevance_scratch_bytes(batch, gamma, n_visual, dim);
+}
+
+size_t lvspec_workspace_capacity(const lvspec_ctx_t *ctx) { return ctx ? ctx->scratch_bytes : 0; }
+
+lvspec_status_t lvspec_reserve(lvspec_ctx_t *ctx, size_t workspace_bytes)
+{
+    if (!ctx) return LVSPEC_ERR_INVALID_ARG;
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
+    return ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, workspace_bytes, false);
 }
 
 lvspec_status_t lvspec_verify_attention(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
@@ -499,7 +582,10 @@ lvspec_status_t lvspec_verify_attention_spans(lvspec_ctx_t *ctx, const lvspec_at
     lvspec_attn_shape_t s = *shape;
     if (resolve_kernel(&s) == LVSPEC_KERNEL_TCGEN05 && s.n_split == 0 && choose_splits(ctx, &s, max_len) < 2) {
         if (max_len > 128) s.n_split = 2;
-        else s.kernel = LVSPEC_KERNEL_SIMT;
+        else if (s.kernel == LVSPEC_KERNEL_DEFAULT) s.kernel = LVSPEC_KERNEL_SIMT;
+        else
+            return fail(ctx, LVSPEC_ERR_UNSUPPORTED,
+                        "several spans on a cache of one tile need the plain kernel (two splits cannot be made)");
     }
     if (resolve_kernel(&s) == LVSPEC_KERNEL_TCGEN05 && s.n_split == 1)
         return fail(ctx, LVSPEC_ERR_UNSUPPORTED, "several spans need n_split != 1 with the tcgen05 kernel");

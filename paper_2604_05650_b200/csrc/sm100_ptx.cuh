@@ -262,24 +262,5 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
-// named barrier over the 128 softmax threads
-__device__ __forceinline__ void wg_sync()
-{
-    asm volatile("bar.sync 1, 128;" ::: "memory");
-}
-__device__ __forceinline__ bool wg_any(bool pred)
-{
-    uint32_t out;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.or.pred p, 1, 128, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(out)
-        : "r"((uint32_t)pred)
-        : "memory");
-    return out != 0;
-}
-
 }  // namespace ptx
 }  // namespace lvspec

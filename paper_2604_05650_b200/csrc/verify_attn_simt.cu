@@ -278,7 +278,11 @@ __global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const 
             const float4 *v = rows + lane;
 #pragma unroll 3
             for (int u = 0; u < n; ++u, v += 32) {
+                // a split without weight (no tile of its own, or all of it masked) may
+                // have left its rows unwritten: whatever the scratch holds there, NaN
+                // bit patterns included, must not reach the sum
                 const float wu = weights[u];
+                if (wu == 0.f) continue;
                 const float4 x = *v;
                 o.x = fmaf(wu, x.x, o.x);
                 o.y = fmaf(wu, x.y, o.y);

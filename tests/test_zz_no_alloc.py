@@ -4,7 +4,8 @@ budgets, loops that must avoid the synchronisation of cudaMalloc).  It keeps
 its scratch in a fixed array inside the library, shared by every call, so the
 check is that two calls in a row, through the C ABI and without any context,
 give exactly what the context-based lvspec_loose_accept gives on the same
-inputs (all outputs are integers: the comparison is bit-exact).
+inputs, and what the CPU oracle gives (all outputs are integers: the
+comparisons are bit-exact).
 
 This file sorts last on purpose: a run that stops at the first failure has
 then already run every other test."""
@@ -22,7 +23,7 @@ def _inputs(cfg, batch):
     return logits, draft, mass
 
 
-def test_two_calls_in_a_row_match_the_context_entry_point():
+def test_two_calls_in_a_row_match_the_context_entry_point(oracle_mod):
     import torch
     from paper_2604_05650_b200 import binding
     assert torch.cuda.is_available(), "GPU tests need a CUDA device"
@@ -59,8 +60,40 @@ def test_two_calls_in_a_row_match_the_context_entry_point():
             torch.cuda.synchronize()
             assert (g == ref.cpu().numpy()).all()
             assert (g >= 0).all() and (g <= cfg.gamma).all()
+            want, _, _ = oracle_mod.loose_accept(logits, draft, mass, oracle_mod.n_loose(cfg.lam, cfg.gamma),
+                                                 window)
+            assert (g == want).all()
     finally:
         ctx.close()
+
+
+def test_most_rows_the_array_takes_and_special_logits(oracle_mod):
+    """batch * gamma = LVSPEC_STATIC_MAX_ROWS: the number of vocabulary slices is then
+    bounded by the array (8 partials per row), not by the device; one row holds a NaN and
+    a -inf logit (NaN ranks as -inf), another nothing above -inf (token 0).  Checked
+    against the oracle directly."""
+    import torch
+    from paper_2604_05650_b200 import binding
+    torch.cuda.set_device(0)
+    batch, gamma, vocab, heads = 128, 8, 40000, 2
+    assert batch * gamma == binding.STATIC_MAX_ROWS
+    rng = np.random.default_rng(4242)
+    logits = rng.standard_normal((batch, gamma, vocab), dtype=np.float32)
+    top = logits.argmax(-1)
+    draft = np.where(rng.random((batch, gamma)) < 0.6, top, rng.integers(0, vocab, (batch, gamma))).astype(np.int32)
+    logits[3, 2, 17] = np.nan
+    logits[3, 2, 31000] = -np.inf
+    logits[5, 0, :] = -np.inf
+    logits[5, 1, :] = np.nan
+    mass = rng.random((batch, gamma, heads), dtype=np.float32)
+    dl, dd, dm = torch.from_numpy(logits).cuda(), torch.from_numpy(draft).cuda(), torch.from_numpy(mass).cuda()
+    for window in (0, 3):
+        alen = torch.full((batch,), -5, dtype=torch.int32, device="cuda")
+        binding.loose_accept_static(torch.cuda.current_stream(), batch, gamma, vocab, heads, dl, dd, dm, alen,
+                                    window, n_loose=3)
+        torch.cuda.synchronize()
+        want, _, _ = oracle_mod.loose_accept(logits, draft, mass, 3, window)
+        assert (alen.cpu().numpy() == want).all()
 
 
 def test_sizes_beyond_the_fixed_array_are_refused():
