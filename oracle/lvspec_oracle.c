@@ -12,7 +12,8 @@
  * attention in fp64 (the attention the paper names in App. "Baseline
  * Details"), closed forms (identical keys, dominant key, key translation),
  * brute-force enumeration and hand-worked cases of the rule (tests/golden),
- * and the closed form of Prop. 2.2.  The paper prints no worked numeric
+ * the closed form of Prop. 2.2, and for the fp8 cache the published E4M3
+ * format through an independent library decoder.  The paper prints no worked numeric
  * example of the rule, so beyond those pins the rule is "parity unpinned"
  * against the authors' own code.
  */
@@ -117,6 +118,92 @@ void lvspec_oracle_verify_attention_tree(const uint16_t *q, const uint16_t *k, c
             if (probs)
                 for (int j = vis > 0 ? vis : 0; j < Lmax; ++j)
                     probs[(((size_t)b * gamma + g) * Hq + h) * (size_t)Lmax + j] = 0.0;
+            mass[((size_t)b * gamma + g) * Hq + h] = vm;
+        }
+        free(s);
+        free(qd);
+    }
+}
+
+/*
+ * An fp8 cache.  The paper's premise is that the target's pass over the long visual
+ * KV cache is bound by memory traffic (Sec. 1; the T_t^K term of the speed-up formula in
+ * Sec. 2.2); storing K and V in 8 bits halves that traffic.  The stored format is the
+ * OCP 8-bit floating point E4M3 ("FN" variant: no infinities): 1 sign bit, 4 exponent
+ * bits with bias 7, 3 mantissa bits;
+ *     exponent field 0:      value = (-1)^s * 2^-6 * (mantissa / 8)            (subnormal)
+ *     otherwise:             value = (-1)^s * 2^(exponent - 7) * (1 + mantissa / 8)
+ *     exponent 15 with mantissa 7 (codes 0x7F, 0xFF) is NaN; the largest finite value is 448.
+ * A cache element is code * scale, with one fp32 scale per (sequence, KV head) for K and
+ * one for V.
+ */
+double lvspec_oracle_e4m3_decode(uint8_t code)
+{
+    const int sign = code >> 7, e = (code >> 3) & 15, m = code & 7;
+    double x;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) x = ldexp((double)m / 8.0, -6);
+    else x = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return sign ? -x : x;
+}
+
+/*
+ * Verification attention with visual mass (Eq. 1; SDPA, App. "Baseline Details") over an
+ * fp8 cache: the plain definition of lvspec_oracle_verify_attention_tree, with every
+ * cache element decoded as above and multiplied by its scale in fp64 first.
+ *
+ *   q           bf16 bits [B, gamma, Hq, D]
+ *   k8, v8      E4M3 codes [B, Hkv, Lmax, D]
+ *   k_scale, v_scale   fp32 [B, Hkv]
+ * everything else as for the bf16 cache.
+ */
+void lvspec_oracle_verify_attention_fp8(const uint16_t *q, const uint8_t *k8, const uint8_t *v8,
+                                        const float *k_scale, const float *v_scale,
+                                        const int32_t *kv_len, const int32_t *span,
+                                        int B, int gamma, int Hq, int Hkv, int D, int Lmax,
+                                        double *out, double *mass)
+{
+    const int G = Hq / Hkv;
+    const double scale = 1.0 / sqrt((double)D);
+    const long units = (long)B * gamma * Hq;
+#pragma omp parallel
+    {
+        double *s = (double *)malloc(sizeof(double) * (size_t)(Lmax > 0 ? Lmax : 1));
+        double *qd = (double *)malloc(sizeof(double) * (size_t)D);
+#pragma omp for schedule(dynamic, 1)
+        for (long u = 0; u < units; ++u) {
+            const int h = (int)(u % Hq);
+            const int g = (int)((u / Hq) % gamma);
+            const int b = (int)(u / ((long)Hq * gamma));
+            const int kvh = h / G;
+            const int vis = kv_len[b] - gamma + g + 1;
+            const int vs = span[2 * b], ve = span[2 * b + 1];
+            const double ks = (double)k_scale[(size_t)b * Hkv + kvh];
+            const double vsc = (double)v_scale[(size_t)b * Hkv + kvh];
+            const uint16_t *qrow = q + (((size_t)b * gamma + g) * Hq + h) * D;
+            const uint8_t *kb = k8 + ((size_t)b * Hkv + kvh) * (size_t)Lmax * D;
+            const uint8_t *vb = v8 + ((size_t)b * Hkv + kvh) * (size_t)Lmax * D;
+            double *orow = out + (((size_t)b * gamma + g) * Hq + h) * D;
+
+            for (int d = 0; d < D; ++d) qd[d] = bf16_to_double(qrow[d]);
+            double m = -INFINITY;
+            for (int j = 0; j < vis; ++j) {
+                double acc = 0.0;
+                for (int d = 0; d < D; ++d) acc += qd[d] * (lvspec_oracle_e4m3_decode(kb[(size_t)j * D + d]) * ks);
+                s[j] = acc * scale;
+                if (s[j] > m) m = s[j];
+            }
+            double Z = 0.0;
+            for (int j = 0; j < vis; ++j) { s[j] = exp(s[j] - m); Z += s[j]; }
+            for (int d = 0; d < D; ++d) orow[d] = 0.0;
+            double vm = 0.0;
+            for (int j = 0; j < vis; ++j) {
+                const double p = s[j] / Z;
+                if (j >= vs && j < ve) vm += p;
+                if (p != 0.0)
+                    for (int d = 0; d < D; ++d)
+                        orow[d] += p * (lvspec_oracle_e4m3_decode(vb[(size_t)j * D + d]) * vsc);
+            }
             mass[((size_t)b * gamma + g) * Hq + h] = vm;
         }
         free(s);

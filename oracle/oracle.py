@@ -43,6 +43,10 @@ def _load():
         lib.lvspec_oracle_verify_attention.restype = None
         lib.lvspec_oracle_verify_attention_tree.argtypes = [p, p, p, p, p, i, i, i, i, i, i, i, p, p, p]
         lib.lvspec_oracle_verify_attention_tree.restype = None
+        lib.lvspec_oracle_verify_attention_fp8.argtypes = [p, p, p, p, p, p, p, i, i, i, i, i, i, p, p]
+        lib.lvspec_oracle_verify_attention_fp8.restype = None
+        lib.lvspec_oracle_e4m3_decode.argtypes = [ctypes.c_uint8]
+        lib.lvspec_oracle_e4m3_decode.restype = ctypes.c_double
         lib.lvspec_oracle_select_branch.argtypes = [p, i, i, p, p]
         lib.lvspec_oracle_select_branch.restype = None
         lib.lvspec_oracle_loose_accept.argtypes = [p, p, p, i, i, i, i, i, i, p, p, p]
@@ -103,6 +107,37 @@ def verify_attention(q, k, v, kv_len, span, return_probs: bool = False, branch_l
                                             B, gamma, bl, Hq, Hkv, D, Lmax, _ptr(out), _ptr(mass),
                                             _ptr(probs))
     return (out, mass, probs) if return_probs else (out, mass)
+
+
+def e4m3_decode(code: int) -> float:
+    """Value of one E4M3 code (0..255)."""
+    return float(_load().lvspec_oracle_e4m3_decode(int(code) & 0xFF))
+
+
+def verify_attention_fp8(q, k8, v8, k_scale, v_scale, kv_len, span):
+    """q [B,gamma,Hq,D] uint16 bf16 bits; k8/v8 [B,Hkv,Lmax,D] uint8 E4M3 codes;
+    k_scale/v_scale fp32 [B,Hkv]; kv_len int32 [B]; span int32 [B,2].
+    Returns (out, mass) in fp64."""
+    lib = _load()
+    q = np.ascontiguousarray(q, dtype=np.uint16)
+    k8 = np.ascontiguousarray(k8, dtype=np.uint8)
+    v8 = np.ascontiguousarray(v8, dtype=np.uint8)
+    k_scale = np.ascontiguousarray(k_scale, dtype=np.float32)
+    v_scale = np.ascontiguousarray(v_scale, dtype=np.float32)
+    kv_len = np.ascontiguousarray(kv_len, dtype=np.int32)
+    span = np.ascontiguousarray(span, dtype=np.int32)
+    B, gamma, Hq, D = q.shape
+    Bk, Hkv, Lmax, Dk = k8.shape
+    assert (Bk, Dk) == (B, D) and v8.shape == k8.shape and Hq % Hkv == 0
+    assert k_scale.shape == (B, Hkv) and v_scale.shape == (B, Hkv)
+    assert kv_len.shape == (B,) and span.shape == (B, 2)
+    assert (kv_len >= gamma).all() and (kv_len <= Lmax).all()
+    out = np.empty((B, gamma, Hq, D), dtype=np.float64)
+    mass = np.empty((B, gamma, Hq), dtype=np.float64)
+    lib.lvspec_oracle_verify_attention_fp8(_ptr(q), _ptr(k8), _ptr(v8), _ptr(k_scale), _ptr(v_scale),
+                                           _ptr(kv_len), _ptr(span), B, gamma, Hq, Hkv, D, Lmax,
+                                           _ptr(out), _ptr(mass))
+    return out, mass
 
 
 def loose_accept(logits, draft, mass, n_loose: int, window: int):

@@ -96,6 +96,42 @@ def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
 
 
 # ----------------------------------------------------------------------------
+# 8-bit storage helper: float32 -> OCP FP8 E4M3 codes (round to nearest even)
+# ----------------------------------------------------------------------------
+def _e4m3_positive_values() -> np.ndarray:
+    """The 127 finite non-negative E4M3 values in code order (0x00..0x7E): exponent
+    field 0 is subnormal, (m/8) 2^-6; otherwise (1 + m/8) 2^(e-7); 0x7F is NaN."""
+    codes = np.arange(127)
+    e, m = codes >> 3, codes & 7
+    return np.where(e == 0, (m / 8.0) * 2.0 ** -6, (1.0 + m / 8.0) * 2.0 ** (e.astype(np.float64) - 7.0))
+
+
+def f32_to_e4m3_bits(x: np.ndarray) -> np.ndarray:
+    """Round float32 values to the nearest E4M3 value (ties to the even code, magnitudes
+    beyond 448 saturate to 448) and return the uint8 codes.  NaN is not expected."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    vals = _e4m3_positive_values()
+    a = np.minimum(np.abs(x).astype(np.float64), 448.0)
+    hi = np.clip(np.searchsorted(vals, a, side="left"), 1, 126)     # vals[hi-1] <= a <= vals[hi] (a > 0)
+    lo = hi - 1
+    d_lo, d_hi = a - vals[lo], vals[hi] - a
+    pick_hi = (d_hi < d_lo) | ((d_hi == d_lo) & ((hi & 1) == 0))
+    code = np.where(pick_hi, hi, lo).astype(np.uint8)
+    return np.where(np.signbit(x), code | np.uint8(0x80), code).astype(np.uint8)
+
+
+def quantize_cache_e4m3(bits: np.ndarray):
+    """A bf16 cache [B, Hkv, L, D] (bit patterns) as an fp8 cache: E4M3 codes of the same
+    shape and one fp32 scale per (sequence, KV head), chosen so that the largest magnitude
+    of that head maps to 448.  Returns (codes uint8, scale float32 [B, Hkv])."""
+    x = bf16_bits_to_f32(bits)
+    amax = np.abs(x).max(axis=(2, 3))
+    scale = (np.where(amax > 0, amax, 1.0) / np.float32(448.0)).astype(np.float32)
+    codes = f32_to_e4m3_bits(x / scale[:, :, None, None])
+    return codes, scale
+
+
+# ----------------------------------------------------------------------------
 # attention inputs
 # ----------------------------------------------------------------------------
 def attention_inputs(cfg: VerifyConfig, layer: int = 0, kv_capacity: int | None = None):
