@@ -106,19 +106,47 @@ int resolve_kernel(const lvspec_attn_shape_t *s)
     return tc_shape(s) ? LVSPEC_KERNEL_TCGEN05 : LVSPEC_KERNEL_SIMT;
 }
 
+// KV splits per (sequence, KV head) when the caller leaves the choice to the library.
+// The tensor-core kernel runs one CTA per SM and is bound by HBM once about three
+// quarters of the SMs stream (one SM alone pulls about 60 GB/s).  Splits are whole
+// 128-position tiles, so a split count that does not divide the tile count leaves a last
+// round in which only the CTAs with one tile more are at work, far below the device's
+// bandwidth: 16 splits of 16 tiles beat 18 splits of 14 or 15 on eight heads of 256 tiles.
+// The count is therefore chosen by a small model of the stream, in units of the time the
+// whole device takes for one tile: the even rounds at the bandwidth their CTA count
+// reaches, the uneven last round at the bandwidth of its few CTAs, and a charge per CTA
+// for writing its partial and merging it.  A pure function of the shape: results stay
+// reproducible from run to run.
 int choose_splits(const lvspec_ctx *ctx, const lvspec_attn_shape_t *s, int max_kv_len)
 {
     const int tiles = (max_kv_len + 127) / 128;           // splits never go below 128 positions
     const int units = s->batch * s->n_kv_heads;
-    int want;
-    if (resolve_kernel(s) == LVSPEC_KERNEL_TCGEN05)
-        want = ctx->n_sm / units;                          // one CTA per SM, one wave
-    else
-        want = (2 * ctx->n_sm + units - 1) / units;        // about two CTAs per SM
-    if (want < 1) want = 1;
-    if (want > tiles) want = tiles;
-    if (want > 256) want = 256;
-    return want;
+    if (resolve_kernel(s) != LVSPEC_KERNEL_TCGEN05) {
+        int want = (2 * ctx->n_sm + units - 1) / units;    // about two CTAs per SM
+        if (want < 1) want = 1;
+        if (want > tiles) want = tiles;
+        if (want > 256) want = 256;
+        return want;
+    }
+    int most = ctx->n_sm / units;                          // one CTA per SM, one wave
+    if (most < 1) most = 1;
+    if (most > tiles) most = tiles;
+    if (most > 256) most = 256;
+    const double saturating = 0.73 * ctx->n_sm;            // CTAs that reach the HBM bandwidth
+    auto rate = [&](double ctas) { return ctas >= saturating ? 1.0 : ctas / saturating; };
+    int best = most;
+    double best_cost = 0.0;
+    for (int ns = most; ns >= 1; --ns) {
+        const double ctas = (double)ns * units;
+        const int t_lo = tiles / ns, rem = tiles - t_lo * ns;
+        double cost = t_lo * ctas / rate(ctas) + 0.7 * ctas;
+        if (rem > 0) cost += (double)rem * units / rate((double)rem * units);
+        if (ns == most || cost < best_cost) {
+            best = ns;
+            best_cost = cost;
+        }
+    }
+    return best;
 }
 
 // Vocabulary slices of the acceptance kernel: enough CTAs for two per SM, at least 4096

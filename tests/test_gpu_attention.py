@@ -257,3 +257,4 @@ def test_plain_launches_give_the_same_results(oracle_mod, monkeypatch):
     ref_out, ref_mass = oracle_mod.verify_attention(*case)
     from gpu_util import assert_attention_close
     assert_attention_close(outs[0][0], outs[0][1], ref_out, ref_mass)
+
