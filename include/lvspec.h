@@ -284,6 +284,35 @@ lvspec_status_t lvspec_verify_attention_paged(lvspec_ctx_t *ctx, const lvspec_at
                                               const int32_t *block_table, const int32_t *kv_len,
                                               const int32_t *visual_span, void *out, float *visual_mass);
 
+/* lvspec_verify_attention on an FP8 cache.  The paper's premise is that the target's
+ * pass over the long visual KV cache is bound by memory traffic (Sec. 1; the T_t^K
+ * term of the speed-up formula in Sec. 2.2): a cache stored in 8 bits halves it.  The
+ * operation is that of Eq. 1 as above, on the cache values
+ *
+ *   k[b,h,j,:] = k_scale[b,h] * decode(k_cache[b,h,j,:]),   v likewise,
+ *
+ * where decode is the OCP 8-bit floating-point format E4M3 (1 sign, 4 exponent bits
+ * with bias 7, 3 mantissa bits; no infinities, codes 0x7F / 0xFF are NaN, largest value
+ * 448):
+ *
+ *   k_cache, v_cache  device, uint8  [B, Hkv, Lmax, D]   E4M3 codes
+ *   k_scale, v_scale  device, fp32   [B, Hkv]            read during the call
+ *
+ * q, out and everything else are as for lvspec_verify_attention (q and out stay bf16).
+ * Arithmetic: the 8-bit tiles go to the tensor cores as they are; q and the
+ * probabilities are each split into two E4M3 terms (leading four significant bits and
+ * the rest) so that they lose no more than they would as bf16; accumulation is fp32.
+ * Probabilities of a row are held within 2^8 above and about 2^11 below those of the
+ * largest score seen so far; terms smaller than that by another factor of 2^6 vanish.
+ * Tolerances against the plain definition on the decoded cache: those of the bf16 call.
+ * UNSUPPORTED for head_dim other than 128, for LVSPEC_KERNEL_SIMT, for more than 80
+ * query rows per KV head (gamma * Hq / Hkv), and for kv_capacity < 128. */
+lvspec_status_t lvspec_verify_attention_fp8(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                            const void *q, const void *k_cache, const void *v_cache,
+                                            const float *k_scale, const float *v_scale,
+                                            const int32_t *kv_len, const int32_t *visual_span,
+                                            void *out, float *visual_mass);
+
 /* Same operation on HOST buffers: copies q, the caches, and the results through
  * device staging memory the context owns (grown on demand), on the context's
  * stream, and synchronises before returning.  All seven arrays are host

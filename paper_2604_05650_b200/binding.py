@@ -34,6 +34,7 @@ EXPORTS = (
     "lvspec_verify_attention_spans", "lvspec_last_device_status",
     "lvspec_attention_workspace_bytes", "lvspec_accept_workspace_bytes",
     "lvspec_relevance_workspace_bytes", "lvspec_workspace_capacity", "lvspec_reserve",
+    "lvspec_verify_attention_fp8",
 )
 
 
@@ -95,6 +96,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lvspec_attention_splits.restype = i32
     lib.lvspec_verify_attention.argtypes = [vp, S, vp, vp, vp, vp, vp, vp, vp]
     lib.lvspec_verify_attention_host.argtypes = [vp, S, vp, vp, vp, vp, vp, vp, vp]
+    lib.lvspec_verify_attention_fp8.argtypes = [vp, S, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.lvspec_loose_accept.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp]
     lib.lvspec_loose_accept_ex.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp, vp, vp]
     lib.lvspec_loose_accept_host.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp]
@@ -211,6 +213,17 @@ class Context:
         self._check(self._lib.lvspec_verify_attention(
             self._h, ctypes.byref(shape), _addr(q), _addr(k_cache), _addr(v_cache),
             kv_len.ctypes.data, span.ctypes.data, _addr(out), _addr(visual_mass)))
+
+    def verify_attention_fp8(self, shape: AttnShape, q, k_cache, v_cache, k_scale, v_scale, kv_len,
+                             visual_span, out, visual_mass) -> None:
+        """k_cache / v_cache: device uint8 E4M3 codes [B, Hkv, Lmax, D]; k_scale / v_scale:
+        device fp32 [B, Hkv]."""
+        kv_len, span = _i32(kv_len), _i32(visual_span)
+        if shape.batch >= 1 and (kv_len.size != shape.batch or span.size != 2 * shape.batch):
+            raise ValueError("kv_len needs B entries and visual_span B pairs")
+        self._check(self._lib.lvspec_verify_attention_fp8(
+            self._h, ctypes.byref(shape), _addr(q), _addr(k_cache), _addr(v_cache), _addr(k_scale),
+            _addr(v_scale), kv_len.ctypes.data, span.ctypes.data, _addr(out), _addr(visual_mass)))
 
     def verify_attention_tree(self, shape: AttnShape, n_branches, q, k_cache, v_cache, kv_len, visual_span,
                               out, visual_mass) -> None:

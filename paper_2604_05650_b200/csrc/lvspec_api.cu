@@ -223,10 +223,14 @@ struct PagedCache {          // page pools instead of one contiguous cache per s
     int page_size = 0, pages_per_seq = 0, n_pages = 0;
 };
 
+struct Fp8Cache {            // E4M3 codes with one scale per (sequence, KV head)
+    const float *k_scale = nullptr, *v_scale = nullptr;
+};
+
 lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, const SeqInfo &seq,
                               int max_len, const void *q, const void *k, const void *v, void *out,
                               float *mass, int branch_len = 0, const PagedCache *paged = nullptr,
-                              float **lse2 = nullptr)
+                              float **lse2 = nullptr, const Fp8Cache *fp8 = nullptr)
 {
     AttnParams p;
     std::memset(&p, 0, sizeof p);
@@ -248,6 +252,11 @@ lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, con
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)p.D));
     p.pdl = ctx->pdl ? 1 : 0;
     p.branch_len = branch_len > 0 ? branch_len : p.gamma;
+    if (fp8) {
+        p.fp8 = 1;
+        p.k_scale = fp8->k_scale;
+        p.v_scale = fp8->v_scale;
+    }
     if (paged) {
         p.block_table = paged->block_table;
         p.page_size = paged->page_size;
@@ -274,7 +283,9 @@ lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, con
     if (kernel == LVSPEC_KERNEL_TCGEN05) {
         if (!attn_tc_supported(p))
             return fail(ctx, LVSPEC_ERR_UNSUPPORTED,
-                        "the tcgen05 kernel needs head_dim 128 and kv_capacity >= 128");
+                        p.fp8 ? "the fp8 cache needs head_dim 128, kv_capacity >= 128 and at most 80 query rows "
+                                "per KV head"
+                              : "the tcgen05 kernel needs head_dim 128 and kv_capacity >= 128");
         e = launch_attn_tc(p, seq, ctx->stream, &launches);
     } else {
         e = launch_attn_simt(p, seq, ctx->stream, &launches);
@@ -684,6 +695,33 @@ lvspec_status_t lvspec_verify_attention_paged(lvspec_ctx_t *ctx, const lvspec_at
     lvspec_attn_shape_t s = *shape;
     s.kernel = LVSPEC_KERNEL_TCGEN05;
     return run_attention(ctx, &s, seq, max_len, q, k_pool, v_pool, out, visual_mass, 0, &pc);
+}
+
+lvspec_status_t lvspec_verify_attention_fp8(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                            const void *q, const void *k_cache, const void *v_cache,
+                                            const float *k_scale, const float *v_scale,
+                                            const int32_t *kv_len, const int32_t *visual_span,
+                                            void *out, float *visual_mass)
+{
+    SeqInfo seq;
+    int max_len = 0;
+    lvspec_status_t st = check_attention(ctx, shape, q, k_cache, v_cache, kv_len, visual_span, out,
+                                         visual_mass, true, &seq, &max_len);
+    if (st != LVSPEC_OK) return st;
+    if (!k_scale || !v_scale || (reinterpret_cast<uintptr_t>(k_scale) & 3u) ||
+        (reinterpret_cast<uintptr_t>(v_scale) & 3u))
+        return fail(ctx, LVSPEC_ERR_INVALID_ARG, "k_scale or v_scale is null or misaligned");
+    if (shape->head_dim != 128 || shape->kernel == LVSPEC_KERNEL_SIMT || shape->kv_capacity < 128)
+        return fail(ctx, LVSPEC_ERR_UNSUPPORTED,
+                    "the fp8 cache needs the tcgen05 kernel (head_dim 128, kv_capacity >= 128)");
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
+    Fp8Cache f8;
+    f8.k_scale = k_scale;
+    f8.v_scale = v_scale;
+    lvspec_attn_shape_t s = *shape;
+    s.kernel = LVSPEC_KERNEL_TCGEN05;
+    return run_attention(ctx, &s, seq, max_len, q, k_cache, v_cache, out, visual_mass, 0, nullptr, nullptr, &f8);
 }
 
 lvspec_status_t lvspec_verify_attention_host(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,

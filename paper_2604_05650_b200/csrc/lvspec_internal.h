@@ -33,6 +33,11 @@ struct AttnParams {
     const int32_t *block_table;
     int32_t page_size, pages_per_seq, n_pages;
     float scale_log2;      // log2(e) / sqrt(D)
+    // fp8 cache (fp8 != 0): k and v point to E4M3 codes, one byte per element, and a
+    // cache element is code * scale with one scale per (sequence, KV head)
+    int32_t fp8;
+    const float *k_scale;  // [B, Hkv]
+    const float *v_scale;  // [B, Hkv]
 };
 
 // Does draft query `qi` see the cache position with tail index t = pos - (kv_len -

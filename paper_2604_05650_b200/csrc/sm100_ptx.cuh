@@ -214,6 +214,17 @@ __device__ __forceinline__ void mma_f16_ss(uint32_t d_tmem, uint64_t a_desc, uin
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// Same for 8-bit floating-point operands (kind::f8f6f4; K = 32 per instruction).
+__device__ __forceinline__ void mma_f8_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                          uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 // The mbarrier receives one arrival when every tcgen05.mma issued so far by
 // this thread has completed.
 __device__ __forceinline__ void mma_commit(uint32_t bar)
@@ -248,6 +259,15 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(uint32_t M, uint32_t N, u
            | (a_mn << 15) | (b_mn << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 
+// Instruction descriptor, kind::f8f6f4: E4M3 x E4M3 -> fp32, dense (operand format
+// code 0 = E4M3 in both fields).
+__host__ __device__ constexpr uint32_t make_idesc_e4m3(uint32_t M, uint32_t N, uint32_t a_mn,
+                                                       uint32_t b_mn)
+{
+    return (1u << 4)            // D format fp32
+           | (a_mn << 15) | (b_mn << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
 // ---- misc ---------------------------------------------------------------------
 __device__ __forceinline__ float ex2(float x)
 {
@@ -262,5 +282,20 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
+// two fp32 -> packed E4M3 pair (lo in the low byte), round to nearest even, saturating
+__device__ __forceinline__ uint32_t pack_e4m3x2(float lo, float hi)
+{
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// The leading four significant bits of an fp32 value (sign, exponent, three mantissa
+// bits: what one E4M3 value holds when the exponent is in its normal range), by
+// truncation; value - head is then exact in fp32.
+__device__ __forceinline__ float e4m3_head(float x)
+{
+    return __uint_as_float(__float_as_uint(x) & 0xFFF00000u);
+}
+
 }  // namespace ptx
 }  // namespace lvspec

@@ -28,6 +28,22 @@
 // each slot two 128-position x 64-channel boxes with the 128-byte swizzle; Q
 // arrives by TMA in the same layout.  Every mbarrier wait is bounded; a wait
 // that gives up raises LVSPEC_DEV_WAIT_EXPIRED.
+//
+// fp8 cache (kFp8): K and V are E4M3 codes with one scale per (sequence, KV head), half
+// the bytes per position.  An MMA takes both operands in one kind, so the 8-bit tiles
+// are multiplied as they are (kind::f8f6f4, K = 32 per instruction) and the bf16
+// side is brought to them without losing its bits: a value is split into the E4M3
+// number holding its leading four significant bits and the E4M3 number nearest to the
+// rest (the next four), both exact for bf16 inputs in the normal range.  Q (scaled by a
+// power of two so that its largest magnitude sits below 256) is split once per CTA into
+// two operand tiles, and K.Q^T takes both in one accumulation (8 MMAs of K = 32 over the
+// 2 x 128 channels); a probability is split by the softmax threads, head and rest sit
+// in neighbouring columns of P^T, and V^T.P^T and the sum products run with N = 2 x
+// rows: accumulator column 2n holds the head's part of row n, column 2n + 1 the rest's,
+// added once in the epilogue.  Probabilities are kept within E4M3's range by holding
+// the reference exponent at most 8 binades below the largest score seen (the first
+// position sits at 2^4).  The K scale folds into the softmax scale, the V scale into the
+// epilogue.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -47,17 +63,22 @@ constexpr int kSoftmaxThreads = 32 * kSoftmaxWarps;
 constexpr int kPvWarp = kSoftmaxWarp0 + kSoftmaxWarps;   // issues the P.V and sum MMAs
 constexpr int kThreads = 32 * (kPvWarp + 1);
 constexpr int kMaxChunks = (LVSPEC_MAX_ROWS / 8 + kSoftmaxGroups - 1) / kSoftmaxGroups;   // per group
-constexpr uint32_t kBoxBytes = 16384;       // 128 positions x 64 channels bf16
-constexpr uint32_t kSlotBytes = 2 * kBoxBytes;
-constexpr uint32_t kA2Bytes = 2048;         // one 64 x 16 constant tile
+constexpr uint32_t kBoxBytes = 16384;       // 128 positions x 64 channels bf16, or x 128 channels E4M3
+constexpr uint32_t kSlotBytes = 2 * kBoxBytes;   // a bf16 tile; an fp8 tile is one box
+constexpr uint32_t kA2Bytes = 2048;         // one 64 x 16 (bf16) or 64 x 32 (E4M3) constant tile
 constexpr float kGuard = 60.f;              // log2 units above m before a rescale
+constexpr float kGuard8 = 8.f;              // fp8 cache: probabilities stay below 2^8 (E4M3 ends at 448)
+constexpr float kHead8 = 5.f;               // fp8 cache: the score a row's reference is taken from has probability 2^5
 constexpr float kMFloor = -1.0e30f;
+constexpr int kQBarrier = 1 + kSoftmaxGroups;   // named barrier over all softmax threads
+constexpr int kMaxRowsFp8 = 80;             // fp8 cache: 6 accumulator columns per padded row in 512
 
 struct TcConfig {
     int n_pad;   // MMA N: rows padded to a multiple of 16
     int ks, vs, pb;   // K slots, V slots, P buffers
     int tmem_cols;
     int page_slots;   // paged cache: pool pages of this split's tiles, one entry per tile
+    int slot_bytes;   // one K or V tile: 32 KB bf16, 16 KB fp8
 };
 
 // Byte offsets of the shared-memory regions (relative to a 1024-aligned base).
@@ -68,8 +89,8 @@ __host__ __device__ inline SmemMap smem_map(const TcConfig &c)
 {
     SmemMap s;
     uint32_t o = 0;
-    s.k = o;    o += c.ks * kSlotBytes;
-    s.v = o;    o += c.vs * kSlotBytes;
+    s.k = o;    o += c.ks * c.slot_bytes;
+    s.v = o;    o += c.vs * c.slot_bytes;
     s.q = o;    o += c.n_pad * 256;
     s.p = o;    o += c.pb * c.n_pad * 256;
     s.a2 = o;   o += 4 * kA2Bytes;
@@ -78,7 +99,7 @@ __host__ __device__ inline SmemMap smem_map(const TcConfig &c)
     s.tmx = o;  o += 4 * c.n_pad * 4;
     s.vis = o;  o += c.n_pad * 8;
     s.bars = o; o += 8 * (2 * c.ks + 2 * c.vs + 4 + 2 * c.pb + 3);
-    s.misc = o; o += 16;
+    s.misc = o; o += 16 + 4 * kSoftmaxWarps;     // TMEM address, abort flag, per-warp maxima of |q|
     s.pages = o; o += 4 * c.page_slots;
     s.total = o;
     return s;
@@ -117,6 +138,38 @@ __device__ __forceinline__ bool group_any(int id, bool pred)
     return out != 0;
 }
 
+// Accumulator values of the 8 rows of column chunk c8 in this warp's lanes: with an fp8
+// cache every row has two columns (the products with the probabilities' leading bits and
+// with the rest), added here.
+template <bool kFp8>
+__device__ __forceinline__ void load_acc8(uint32_t taddr, int c8, float (&v)[8])
+{
+    if (kFp8) {
+        uint32_t a[8], b[8];
+        tmem_ld_x8(taddr + c8 * 16, a);
+        tmem_ld_x8(taddr + c8 * 16 + 8, b);
+        tmem_wait_ld();
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            v[k] = __uint_as_float(a[2 * k]) + __uint_as_float(a[2 * k + 1]);
+            v[4 + k] = __uint_as_float(b[2 * k]) + __uint_as_float(b[2 * k + 1]);
+        }
+    } else {
+        uint32_t a[8];
+        tmem_ld_x8(taddr + c8 * 8, a);
+        tmem_wait_ld();
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[k] = __uint_as_float(a[k]);
+    }
+}
+
+template <bool kFp8>
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc)
+{
+    if (kFp8) mma_f8_ss(d, a, b, idesc, acc);
+    else mma_f16_ss(d, a, b, idesc, acc);
+}
+
 // Which draft slots a column's query sees: tail indices [lo, hi] (its own branch up to
 // itself); the context before the draft slots (tail index < 0) is visible to all.
 __device__ __forceinline__ bool column_sees(int2 lohi, int t)
@@ -127,7 +180,9 @@ __device__ __forceinline__ bool column_sees(int2 lohi, int t)
 // exp2 of eight scaled scores of one position, packed to bf16; returns their maximum
 // kMask: 0 = every column sees the position; 1 = plain chain of draft tokens (query
 // col / G sees tail index t iff it is not below t); 2 = draft tree (table look-up)
-template <int kMask>
+// kFp8: each probability goes out as two E4M3 values in neighbouring bytes, its leading
+// four significant bits and the rest (see the head of this file).
+template <int kMask, bool kFp8>
 __device__ __forceinline__ float exp_chunk(const uint32_t (&r)[8], const float *m8, float scale,
                                            const int2 *vis8, int col0, int G, int t, uint4 &dst)
 {
@@ -147,10 +202,24 @@ __device__ __forceinline__ float exp_chunk(const uint32_t (&r)[8], const float *
     float mx = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])),
                      fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
     uint4 pk;
-    pk.x = pack_bf16x2(ex2(x[0]), ex2(x[1]));
-    pk.y = pack_bf16x2(ex2(x[2]), ex2(x[3]));
-    pk.z = pack_bf16x2(ex2(x[4]), ex2(x[5]));
-    pk.w = pack_bf16x2(ex2(x[6]), ex2(x[7]));
+    if (kFp8) {
+        uint32_t w[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const float pr = ex2(x[k]);
+            const float hd = e4m3_head(pr);
+            w[k] = pack_e4m3x2(hd, pr - hd);
+        }
+        pk.x = w[0] | (w[1] << 16);
+        pk.y = w[2] | (w[3] << 16);
+        pk.z = w[4] | (w[5] << 16);
+        pk.w = w[6] | (w[7] << 16);
+    } else {
+        pk.x = pack_bf16x2(ex2(x[0]), ex2(x[1]));
+        pk.y = pack_bf16x2(ex2(x[2]), ex2(x[3]));
+        pk.z = pack_bf16x2(ex2(x[4]), ex2(x[5]));
+        pk.w = pack_bf16x2(ex2(x[6]), ex2(x[7]));
+    }
     dst = pk;
     return mx;
 }
@@ -159,7 +228,7 @@ __device__ __forceinline__ float exp_chunk(const uint32_t (&r)[8], const float *
 // four TMEM loads in flight per wait), packed probabilities into pk, returns the
 // largest scaled score.  kMask != 0: the tile reaches into the draft slots, so
 // columns are masked by what their query may see; the common tile carries none of that.
-template <int kMask>
+template <int kMask, bool kFp8>
 __device__ __forceinline__ float softmax_pass(uint32_t s_addr, int c_lo, int c_hi, const float *m_s,
                                               float scale, const int2 *vis_s, int G, int t,
                                               uint4 (&pk)[kMaxChunks])
@@ -177,8 +246,8 @@ __device__ __forceinline__ float softmax_pass(uint32_t s_addr, int c_lo, int c_h
 #pragma unroll
             for (int u = 0; u < 4; ++u)
                 if (4 * h + u < kMaxChunks && cb + u < c_hi)
-                    gmax = fmaxf(gmax, exp_chunk<kMask>(r[u], m_s + (cb + u) * 8, scale, vis_s + (cb + u) * 8,
-                                                        (cb + u) * 8, G, t, pk[4 * h + u]));
+                    gmax = fmaxf(gmax, exp_chunk<kMask, kFp8>(r[u], m_s + (cb + u) * 8, scale, vis_s + (cb + u) * 8,
+                                                              (cb + u) * 8, G, t, pk[4 * h + u]));
         }
     }
     return gmax;
@@ -187,11 +256,13 @@ __device__ __forceinline__ float softmax_pass(uint32_t s_addr, int c_lo, int c_h
 // kTree: the draft slots hold several branches (the visibility table is only built
 // and read then; the plain chain keeps its arithmetic mask).  kPaged: K and V are page
 // pools and a tile's position in them comes from the sequence's block table.
-template <bool kTree, bool kPaged>
+// kFp8: E4M3 cache (tmap_q is not used: q is split into its two E4M3 tiles by the CTA).
+template <bool kTree, bool kPaged, bool kFp8>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUtensorMap tmap_k,
                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_q)
 {
+    constexpr uint32_t kSlot = kFp8 ? kBoxBytes : kSlotBytes;   // bytes of one K or V tile
     extern __shared__ uint8_t smem_raw[];
     const AttnParams &p = P.a;
     const TcConfig cfg = P.cfg;
@@ -201,7 +272,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     // load is what the whole CTA waits for)
     if (warp == kPvWarp) {
         if (lane == 0) prefetch_tensormap(&tmap_k);
-        if (lane == 1) prefetch_tensormap(&tmap_q);
+        if (lane == 1 && !kFp8) prefetch_tensormap(&tmap_q);
         if (lane == 2) prefetch_tensormap(&tmap_v);
     }
     const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
@@ -272,19 +343,21 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         const int ks = i % cfg.ks;
         int pos0, map_row;
         tile_at(i, pos0, map_row);
-        mbar_arrive_expect_tx(k_full(ks), kSlotBytes);
-        tma_load_3d_hint(base + sm.k + ks * kSlotBytes, &tmap_k, k_full(ks), 0, pos0, map_row, stream_policy);
-        tma_load_3d_hint(base + sm.k + ks * kSlotBytes + kBoxBytes, &tmap_k, k_full(ks), 64, pos0, map_row,
-                         stream_policy);
+        mbar_arrive_expect_tx(k_full(ks), kSlot);
+        tma_load_3d_hint(base + sm.k + ks * kSlot, &tmap_k, k_full(ks), 0, pos0, map_row, stream_policy);
+        if (!kFp8)
+            tma_load_3d_hint(base + sm.k + ks * kSlot + kBoxBytes, &tmap_k, k_full(ks), 64, pos0, map_row,
+                             stream_policy);
     };
     auto load_v = [&](int i) {
         const int vsl = i % cfg.vs;
         int pos0, map_row;
         tile_at(i, pos0, map_row);
-        mbar_arrive_expect_tx(v_full(vsl), kSlotBytes);
-        tma_load_3d_hint(base + sm.v + vsl * kSlotBytes, &tmap_v, v_full(vsl), 0, pos0, map_row, stream_policy);
-        tma_load_3d_hint(base + sm.v + vsl * kSlotBytes + kBoxBytes, &tmap_v, v_full(vsl), 64, pos0, map_row,
-                         stream_policy);
+        mbar_arrive_expect_tx(v_full(vsl), kSlot);
+        tma_load_3d_hint(base + sm.v + vsl * kSlot, &tmap_v, v_full(vsl), 0, pos0, map_row, stream_policy);
+        if (!kFp8)
+            tma_load_3d_hint(base + sm.v + vsl * kSlot + kBoxBytes, &tmap_v, v_full(vsl), 64, pos0, map_row,
+                             stream_policy);
     };
 
     // ------------------------------------------------------------------ prologue
@@ -298,12 +371,13 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             // s_full[2], s_free[2], p_full, p_free, drain, done, q_full
             const int n_kv = 2 * cfg.ks + 2 * cfg.vs;
             const int n_bars = n_kv + 4 + 2 * cfg.pb + 3;
-            if (lane < n_bars) {
-                const int j = lane - n_kv;       // index among the barriers after the rings
+            for (int i = lane; i < n_bars; i += 32) {
+                const int j = i - n_kv;          // index among the barriers after the rings
                 uint32_t count = 1;
                 if (j >= 2 && j < 4 + cfg.pb) count = kSoftmaxWarps;           // s_free, p_full
                 else if (j == 4 + 2 * cfg.pb + 1) count = kSoftmaxWarps + 1;   // done
-                mbar_init(bar0 + 8 * lane, count);
+                else if (kFp8 && j == 4 + 2 * cfg.pb + 2) count = kSoftmaxWarps;   // q_full: the warps that split q
+                mbar_init(bar0 + 8 * i, count);
             }
             if (lane == 0) *abort_flag = 0;
             mbar_fence_init();
@@ -325,9 +399,11 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             first_k = min(T, cfg.ks);
             first_v = min(T, cfg.vs);
             load_k(0);
-            mbar_arrive_expect_tx(q_full, (uint32_t)M * 256u);
-            tma_load_4d(base + sm.q, &tmap_q, q_full, 0, kvh * G, 0, b);
-            tma_load_4d(base + sm.q + NP * 128, &tmap_q, q_full, 64, kvh * G, 0, b);
+            if (!kFp8) {
+                mbar_arrive_expect_tx(q_full, (uint32_t)M * 256u);
+                tma_load_4d(base + sm.q, &tmap_q, q_full, 0, kvh * G, 0, b);
+                tma_load_4d(base + sm.q + NP * 128, &tmap_q, q_full, 64, kvh * G, 0, b);
+            }
             for (int i = 0; i < first_v; ++i) {
                 if (i > 0 && i < first_k) load_k(i);
                 load_v(i);
@@ -339,8 +415,9 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         tmem_relinquish();
     } else if (warp < kPvWarp) {
         const int idx = tid - 64;   // 0..kSoftmaxThreads-1
-        // rows M..NP-1 of Q are padding: zero them (the TMA boxes cover rows < M only)
-        for (int i = idx; i < (NP - M) * 16; i += kSoftmaxThreads) {
+        // rows M..NP-1 of Q are padding: zero them (the TMA boxes cover rows < M only;
+        // with an fp8 cache the split of q below writes every row)
+        for (int i = idx; !kFp8 && i < (NP - M) * 16; i += kSoftmaxThreads) {
             const int r = M + (i >> 4), c = i & 15, h = c >> 3, cc = c & 7;
             *reinterpret_cast<uint4 *>(gbase + sm.q + h * (NP * 128) + r * 128 + cc * 16) =
                 make_uint4(0, 0, 0, 0);
@@ -349,7 +426,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         for (uint32_t i = idx * 16; i < (uint32_t)(cfg.pb * NP * 256); i += kSoftmaxThreads * 16)
             *reinterpret_cast<uint4 *>(gbase + sm.p + i) = make_uint4(0, 0, 0, 0);
         for (int n = idx; n < NP; n += kSoftmaxThreads) {
-            m_s[n] = 0.f;
+            m_s[n] = kFp8 ? kMFloor : 0.f;
             if (kTree) {
                 // the draft slots column n's query sees: its branch's first slot .. its own slot
                 const int qi = n / G;
@@ -362,29 +439,30 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         // l), row 1 = 1 inside the visual span (sums l_vis), rows 2.. = 0.
         // tile 0: block inside the span, 1: outside, 2: the 16-block holding the
         // span start, 3: the 16-block holding the span end
+        // (fp8 cache: the tiles are 64 x 32 E4M3, 16 positions per 16-byte chunk, and the
+        // boundary tiles cover the 32-block holding the span's start / end)
         for (uint32_t i = idx * 16; i < 4 * kA2Bytes; i += kSoftmaxThreads * 16) {
             const int tile = i / kA2Bytes, off = i % kA2Bytes;
             const int c = off / 1024, rr = (off % 1024) / 16;   // rr = row index 0..63
             uint4 val = make_uint4(0, 0, 0, 0);
             if (rr < 2) {
-                uint16_t e[8];
+                constexpr int kPer = kFp8 ? 16 : 8;             // positions per 16-byte chunk
+                uint32_t w[4] = {0, 0, 0, 0};
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
+                for (int k = 0; k < kPer; ++k) {
                     int ind = 1;
                     if (rr == 1) {
                         if (tile == 0) ind = 1;
                         else if (tile == 1) ind = 0;
                         else {
-                            const int pos = ((tile == 2 ? vs : ve) & ~15) + c * 8 + k;
+                            const int pos = ((tile == 2 ? vs : ve) & ~(2 * kPer - 1)) + c * kPer + k;
                             ind = (pos >= vs && pos < ve) ? 1 : 0;
                         }
                     }
-                    e[k] = ind ? 0x3F80 : 0;
+                    if (kFp8) w[k >> 2] |= (ind ? 0x38u : 0u) << (8 * (k & 3));       // E4M3 1.0
+                    else w[k >> 1] |= (ind ? 0x3F80u : 0u) << (16 * (k & 1));         // bf16 1.0
                 }
-                val.x = e[0] | ((uint32_t)e[1] << 16);
-                val.y = e[2] | ((uint32_t)e[3] << 16);
-                val.z = e[4] | ((uint32_t)e[5] << 16);
-                val.w = e[6] | ((uint32_t)e[7] << 16);
+                val = make_uint4(w[0], w[1], w[2], w[3]);
             }
             *reinterpret_cast<uint4 *>(gbase + sm.a2 + i) = val;
         }
@@ -396,7 +474,78 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tm_s0 = tmem_base, tm_o = tmem_base + 2 * NP, tm_l = tmem_base + 3 * NP;
+    // accumulator columns: S^T twice, then O^T and the sums (fp8 cache: two columns per row)
+    constexpr int kAccCols = kFp8 ? 2 : 1;
+    const uint32_t tm_s0 = tmem_base, tm_o = tmem_base + 2 * NP, tm_l = tm_o + kAccCols * NP;
+    float scale_cta = p.scale_log2;     // softmax scale of this CTA (fp8 cache: with the K scale and q's shift)
+    float v_scale = 1.f;
+    if (kFp8 && warp >= kSoftmaxWarp0 && warp < kPvWarp) {
+        // ---- q as two E4M3 operand tiles (128-byte swizzle, one 128-byte row per query row)
+        // chunk = 8 channels of one row (16 bytes of bf16 in, 8 + 8 bytes out)
+        const int idx = tid - 32 * kSoftmaxWarp0;
+        const int n_chunks = NP * 16;
+        constexpr int kMine = (kMaxRowsFp8 * 16 + kSoftmaxThreads - 1) / kSoftmaxThreads;
+        uint4 qv[kMine];
+        float amax = 0.f;
+#pragma unroll
+        for (int u = 0; u < kMine; ++u) {
+            const int ch = idx + u * kSoftmaxThreads;
+            qv[u] = make_uint4(0, 0, 0, 0);
+            if (ch < n_chunks) {
+                const int n = ch >> 4, c = ch & 15;
+                if (n < M) {
+                    const int g = n / G, hg = n - g * G;
+                    qv[u] = __ldg(reinterpret_cast<const uint4 *>(
+                        p.q + (((size_t)b * gamma + g) * p.Hq + kvh * G + hg) * 128 + c * 8));
+                }
+                const uint32_t w[4] = {qv[u].x, qv[u].y, qv[u].z, qv[u].w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    amax = fmaxf(amax, fabsf(__uint_as_float(w[k] << 16)));
+                    amax = fmaxf(amax, fabsf(__uint_as_float(w[k] & 0xFFFF0000u)));
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        volatile float *wmax = reinterpret_cast<volatile float *>(gbase + sm.misc + 16);
+        if (lane == 0) wmax[warp - kSoftmaxWarp0] = amax;
+        asm volatile("bar.sync %0, %1;" ::"r"(kQBarrier), "r"(kSoftmaxThreads) : "memory");
+        amax = 0.f;
+#pragma unroll
+        for (int u = 0; u < kSoftmaxWarps; ++u) amax = fmaxf(amax, wmax[u]);
+        // power of two that brings the largest magnitude into [128, 256) (NaN or Inf in q:
+        // no shift; the result is then NaN as it would be with any cache)
+        int shift = 0;
+        if (amax > 0.f && amax < INFINITY) shift = 7 - ((int)((__float_as_uint(amax) >> 23) & 0xFF) - 127);
+        shift = max(-100, min(100, shift));
+        const float up = __uint_as_float((uint32_t)(127 + shift) << 23);
+#pragma unroll
+        for (int u = 0; u < kMine; ++u) {
+            const int ch = idx + u * kSoftmaxThreads;
+            if (ch < n_chunks) {
+                const int n = ch >> 4, c = ch & 15;
+                const uint32_t w[4] = {qv[u].x, qv[u].y, qv[u].z, qv[u].w};
+                uint32_t hd[4], rs[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float x0 = __uint_as_float(w[k] << 16) * up, x1 = __uint_as_float(w[k] & 0xFFFF0000u) * up;
+                    const float h0 = e4m3_head(x0), h1 = e4m3_head(x1);
+                    hd[k] = pack_e4m3x2(h0, h1);
+                    rs[k] = pack_e4m3x2(x0 - h0, x1 - h1);
+                }
+                const uint32_t off = n * 128 + (((c >> 1) ^ (n & 7)) << 4) + ((c & 1) << 3);
+                *reinterpret_cast<uint2 *>(gbase + sm.q + off) = make_uint2(hd[0] | (hd[1] << 16), hd[2] | (hd[3] << 16));
+                *reinterpret_cast<uint2 *>(gbase + sm.q + NP * 128 + off) =
+                    make_uint2(rs[0] | (rs[1] << 16), rs[2] | (rs[3] << 16));
+            }
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(q_full);
+        scale_cta = p.scale_log2 * __ldg(p.k_scale + bh) * __uint_as_float((uint32_t)(127 - shift) << 23);
+        v_scale = __ldg(p.v_scale + bh);
+    }
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -443,7 +592,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            const uint32_t idesc_qk = make_idesc_bf16(128, NP, 0, 0);
+            const uint32_t idesc_qk = kFp8 ? make_idesc_e4m3(128, NP, 0, 0) : make_idesc_bf16(128, NP, 0, 0);
             // descriptors: everything but the start address is fixed, and the start
             // address field (address / 16) moves by compile-time steps
             const uint64_t kd0 = make_smem_desc(base + sm.k, 16, 1024, kSwizzle128B);
@@ -457,12 +606,16 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 if (!mbar_wait(k_full(ks), (i / cfg.ks) & 1, abort_flag)) return false;
                 if (i >= 2 && !mbar_wait(s_free(sb), ((i >> 1) - 1) & 1, abort_flag)) return false;
                 tc_fence_after();
-                const uint64_t kd = kd0 + (uint64_t)(ks * (kSlotBytes >> 4));
+                const uint64_t kd = kd0 + (uint64_t)(ks * (kSlot >> 4));
                 const uint32_t d = tm_s0 + sb * NP;
+                // bf16: 8 steps of 16 channels over the two 64-channel boxes; fp8: 4 steps of
+                // 32 channels against q's leading bits, then the same 4 against the rest
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    mma_f16_ss(d, kd + (uint64_t)((j >> 2) * (kBoxBytes >> 4) + (j & 3) * 2), qd[j],
-                               idesc_qk, j > 0);
+                for (int j = 0; j < 8; ++j) {
+                    if (kFp8) mma_f8_ss(d, kd + (uint64_t)((j & 3) * 2), qd[j], idesc_qk, j > 0);
+                    else mma_f16_ss(d, kd + (uint64_t)((j >> 2) * (kBoxBytes >> 4) + (j & 3) * 2), qd[j],
+                                    idesc_qk, j > 0);
+                }
                 mma_commit(s_full(sb));
                 mma_commit(k_empty(ks));
                 return true;
@@ -476,8 +629,11 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     } else if (warp == kPvWarp) {
         // ------------------------------------------------- P.V and sum MMA issuer
         if (lane == 0) {
-            const uint32_t idesc_pv = make_idesc_bf16(128, NP, 1, 1);
-            const uint32_t idesc_sum = make_idesc_bf16(64, NP, 0, 1);
+            const uint32_t idesc_pv = kFp8 ? make_idesc_e4m3(128, 2 * NP, 1, 1) : make_idesc_bf16(128, NP, 1, 1);
+            const uint32_t idesc_sum = kFp8 ? make_idesc_e4m3(64, 2 * NP, 0, 1) : make_idesc_bf16(64, NP, 0, 1);
+            // one MMA covers 16 positions of a bf16 tile, 32 of an fp8 tile
+            constexpr int kSteps = kFp8 ? 4 : 8, kStepPos = kTilePos / kSteps;
+            constexpr uint32_t kVStep = kStepPos * 128 >> 4, kPStep = kStepPos * 16 >> 4;   // descriptor units
             const uint64_t vd0 = make_smem_desc(base + sm.v, kBoxBytes, 1024, kSwizzle128B);
             const uint64_t pd0 = make_smem_desc(base + sm.p, 128, 2048, kSwizzleNone);
             const uint64_t a2d0 = make_smem_desc(base + sm.a2, 1024, 128, kSwizzleNone);
@@ -490,11 +646,11 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 // groups of 8 positions 1024 bytes apart.  P^T: rows contiguous in
                 // 16-byte chunks (N-major), chunk stride 2048, groups of 8 positions 128
                 // bytes apart.
-                const uint64_t vd = vd0 + (uint64_t)(vsl * (kSlotBytes >> 4));
+                const uint64_t vd = vd0 + (uint64_t)(vsl * (kSlot >> 4));
                 const uint64_t pd = pd0 + (uint64_t)(pb * ((NP * 256) >> 4));
                 const int pos0 = (t_begin + i) * kTilePos;
-                // constant tile per block of 16 positions: 0 inside the span, 1 outside,
-                // 2 / 3 the blocks holding the span's start / end
+                // constant tile per block of 16 (fp8: 32) positions: 0 inside the span, 1
+                // outside, 2 / 3 the blocks holding the span's start / end
                 int uniform = -1;
                 if (pos0 >= vs && pos0 + kTilePos <= ve) uniform = 0;
                 else if (pos0 + kTilePos <= vs || pos0 >= ve) uniform = 1;
@@ -502,25 +658,25 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 if (uniform >= 0) {
                     const uint64_t d2 = a2d0 + (uint64_t)(uniform * (kA2Bytes >> 4));
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        mma_f16_ss(tm_l, d2, pd + (uint64_t)(j * 16), idesc_sum, j > 0 ? 1u : first_acc);
+                    for (int j = 0; j < kSteps; ++j)
+                        mma_ss<kFp8>(tm_l, d2, pd + (uint64_t)(j * kPStep), idesc_sum, j > 0 ? 1u : first_acc);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        mma_f16_ss(tm_o, vd + (uint64_t)(j * 128), pd + (uint64_t)(j * 16), idesc_pv,
-                                   j > 0 ? 1u : first_acc);
+                    for (int j = 0; j < kSteps; ++j)
+                        mma_ss<kFp8>(tm_o, vd + (uint64_t)(j * kVStep), pd + (uint64_t)(j * kPStep), idesc_pv,
+                                     j > 0 ? 1u : first_acc);
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
+                    for (int j = 0; j < kSteps; ++j) {
                         const uint32_t acc = j > 0 ? 1u : first_acc;
-                        const int pblk = pos0 + 16 * j;
+                        const int pblk = pos0 + kStepPos * j;
                         int tile;
-                        if (pblk >= vs && pblk + 16 <= ve) tile = 0;
-                        else if (pblk + 16 <= vs || pblk >= ve) tile = 1;
-                        else if ((vs & ~15) == pblk) tile = 2;
+                        if (pblk >= vs && pblk + kStepPos <= ve) tile = 0;
+                        else if (pblk + kStepPos <= vs || pblk >= ve) tile = 1;
+                        else if ((vs & ~(kStepPos - 1)) == pblk) tile = 2;
                         else tile = 3;
-                        mma_f16_ss(tm_o, vd + (uint64_t)(j * 128), pd + (uint64_t)(j * 16), idesc_pv, acc);
-                        mma_f16_ss(tm_l, a2d0 + (uint64_t)(tile * (kA2Bytes >> 4)),
-                                   pd + (uint64_t)(j * 16), idesc_sum, acc);
+                        mma_ss<kFp8>(tm_o, vd + (uint64_t)(j * kVStep), pd + (uint64_t)(j * kPStep), idesc_pv, acc);
+                        mma_ss<kFp8>(tm_l, a2d0 + (uint64_t)(tile * (kA2Bytes >> 4)),
+                                     pd + (uint64_t)(j * kPStep), idesc_sum, acc);
                     }
                 }
                 mma_commit(v_empty(vsl));
@@ -540,7 +696,9 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         // chunks of 8 columns [c_lo, c_hi) of this group: equal shares, at most kMaxChunks
         const int c_base = n8 / kSoftmaxGroups, c_rem = n8 - c_base * kSoftmaxGroups;
         const int c_lo = grp * c_base + min(grp, c_rem), c_hi = c_lo + c_base + (grp < c_rem ? 1 : 0);
-        const float scale = p.scale_log2;
+        const float scale = scale_cta;
+        constexpr float kLimit = kFp8 ? kGuard8 : kGuard;    // a score this far above m moves m
+        constexpr float kLift = kFp8 ? kHead8 : 0.f;         // where the reference position sits above m
         // ring positions advance by counting, not by dividing
         int pb = 0, vsl = 0;                 // P buffer and V slot of tile i
         uint32_t pb_round = 0, vs_round = 0; // how often each ring has wrapped
@@ -551,7 +709,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             mbar_wait(s_full(sb), (i >> 1) & 1, abort_flag);
             tc_fence_after();
             const uint32_t s_addr = tm_s0 + sb * NP + lane_addr;
-            if (i == 0) {
+            if (!kFp8 && i == 0) {
                 // reference exponent of each row: its score at the split's first position
                 if (wq == 0) {
                     for (int c8 = c_lo; c8 < c_hi; ++c8) {
@@ -560,7 +718,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                         tmem_wait_ld();
                         if (lane == 0) {
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) m_s[c8 * 8 + k] = __uint_as_float(r[k]) * scale;
+                            for (int k = 0; k < 8; ++k) m_s[c8 * 8 + k] = __uint_as_float(r[k]) * scale - kLift;
                         }
                     }
                 }
@@ -572,10 +730,16 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             uint4 pk[kMaxChunks];   // this position's probabilities, 8 columns per entry
 
             for (int attempt = 0; attempt < 3; ++attempt) {
-                const float gmax =
-                    !tail ? softmax_pass<0>(s_addr, c_lo, c_hi, m_s, scale, vis_s, G, gmin, pk)
-                          : softmax_pass<kTree ? 2 : 1>(s_addr, c_lo, c_hi, m_s, scale, vis_s, G, gmin, pk);
-                if (!group_any(bar_id, gmax > kGuard)) break;
+                // fp8 cache: E4M3 has 17 binades, so the reference exponent of a row starts
+                // from the largest score of the split's first tile (the path below), not
+                // from whatever score its first position happens to have
+                const bool first_max = kFp8 && i == 0 && attempt == 0;
+                if (!first_max) {
+                    const float gmax =
+                        !tail ? softmax_pass<0, kFp8>(s_addr, c_lo, c_hi, m_s, scale, vis_s, G, gmin, pk)
+                              : softmax_pass<kTree ? 2 : 1, kFp8>(s_addr, c_lo, c_hi, m_s, scale, vis_s, G, gmin, pk);
+                    if (!group_any(bar_id, gmax > kLimit)) break;
+                }
 
                 // ---- a score ran past the guard: move m up to the tile maximum ----
                 for (int c8 = c_lo; c8 < c_hi; ++c8) {
@@ -596,7 +760,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 group_sync(bar_id);
                 for (int n = c_lo * 8 + gtid; n < c_hi * 8; n += 128) {
                     const float mt = fmaxf(fmaxf(tmx_s[n], tmx_s[NP + n]),
-                                           fmaxf(tmx_s[2 * NP + n], tmx_s[3 * NP + n]));
+                                           fmaxf(tmx_s[2 * NP + n], tmx_s[3 * NP + n])) - kLift;
                     const float mo = m_s[n];
                     const float mn = fmaxf(mo, mt);
                     dl_s[n] = mo - mn;              // <= 0
@@ -613,21 +777,22 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                         mbar_wait(p_free(pp), pr & 1, abort_flag);
                     }
                     tc_fence_after();
-                    for (int c8 = c_lo; c8 < c_hi; ++c8) {
+                    // (fp8 cache: accumulator columns 2n and 2n + 1 belong to row n)
+                    for (int c = c_lo * kAccCols; c < c_hi * kAccCols; ++c) {
                         uint32_t r[8];
-                        tmem_ld_x8(tm_o + lane_addr + c8 * 8, r);
+                        tmem_ld_x8(tm_o + lane_addr + c * 8, r);
                         tmem_wait_ld();
 #pragma unroll
                         for (int k = 0; k < 8; ++k)
-                            r[k] = __float_as_uint(__uint_as_float(r[k]) * ex2(dl_s[c8 * 8 + k]));
-                        tmem_st_x8(tm_o + lane_addr + c8 * 8, r);
+                            r[k] = __float_as_uint(__uint_as_float(r[k]) * ex2(dl_s[(c * 8 + k) / kAccCols]));
+                        tmem_st_x8(tm_o + lane_addr + c * 8, r);
                         if (wq == 0) {
-                            tmem_ld_x8(tm_l + c8 * 8, r);
+                            tmem_ld_x8(tm_l + c * 8, r);
                             tmem_wait_ld();
 #pragma unroll
                             for (int k = 0; k < 8; ++k)
-                                r[k] = __float_as_uint(__uint_as_float(r[k]) * ex2(dl_s[c8 * 8 + k]));
-                            tmem_st_x8(tm_l + c8 * 8, r);
+                                r[k] = __float_as_uint(__uint_as_float(r[k]) * ex2(dl_s[(c * 8 + k) / kAccCols]));
+                            tmem_st_x8(tm_l + c * 8, r);
                         }
                     }
                     tmem_wait_st();
@@ -640,11 +805,11 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 // rows so that 0 * junk cannot poison the accumulators
                 mbar_wait(v_full(vsl), vs_round & 1, abort_flag);
                 if (pos >= L) {
-                    uint8_t *vrow = gbase + sm.v + vsl * kSlotBytes + row * 128;
+                    uint8_t *vrow = gbase + sm.v + vsl * kSlot + row * 128;
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         *reinterpret_cast<uint4 *>(vrow + c * 16) = make_uint4(0, 0, 0, 0);
-                        *reinterpret_cast<uint4 *>(vrow + kBoxBytes + c * 16) = make_uint4(0, 0, 0, 0);
+                        if (!kFp8) *reinterpret_cast<uint4 *>(vrow + kBoxBytes + c * 16) = make_uint4(0, 0, 0, 0);
                     }
                 }
             }
@@ -677,16 +842,15 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             // a single split: nothing to merge, normalise and write the results here
             if (wq == 0) {
                 for (int c8 = c_lo; c8 < c_hi; ++c8) {
-                    uint32_t r[8];
-                    tmem_ld_x8(tm_l + c8 * 8, r);     // lane 0: l, lane 1: l_vis
-                    tmem_wait_ld();
+                    float lsum[8];
+                    load_acc8<kFp8>(tm_l, c8, lsum);      // lane 0: l, lane 1: l_vis
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
                         const int n = c8 * 8 + k;
-                        const float lv = __shfl_sync(0xffffffffu, __uint_as_float(r[k]), 1);
+                        const float lv = __shfl_sync(0xffffffffu, lsum[k], 1);
                         if (lane == 0 && n < M) {
-                            const float inv = 1.f / __uint_as_float(r[k]);
-                            dl_s[n] = inv;
+                            const float inv = 1.f / lsum[k];
+                            dl_s[n] = inv * v_scale;
                             const int g = n / G, hg = n - g * G;
                             p.mass[((size_t)b * gamma + g) * p.Hq + kvh * G + hg] = lv * inv;
                         }
@@ -696,16 +860,15 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             group_sync(bar_id);
             __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(p.out);
             for (int c8 = c_lo; c8 < c_hi; ++c8) {
-                uint32_t r[8];
-                tmem_ld_x8(tm_o + lane_addr + c8 * 8, r);
-                tmem_wait_ld();
+                float o8[8];
+                load_acc8<kFp8>(tm_o + lane_addr, c8, o8);
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
                     const int n = c8 * 8 + k;
                     if (n < M) {
                         const int g = n / G, hg = n - g * G;
                         out[(((size_t)b * gamma + g) * p.Hq + kvh * G + hg) * 128 + row] =
-                            __float2bfloat16_rn(__uint_as_float(r[k]) * dl_s[n]);
+                            __float2bfloat16_rn(o8[k] * dl_s[n]);
                     }
                 }
             }
@@ -716,30 +879,32 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             float *po = part_o + (size_t)c_lo * 8 * 128 + row;
 #pragma unroll 1
             for (int c8 = c_lo; c8 < c_hi; ++c8, po += 8 * 128) {
-                uint32_t r[8];
-                tmem_ld_x8(tm_o + lane_addr + c8 * 8, r);
-                tmem_wait_ld();
+                float o8[8];
+                load_acc8<kFp8>(tm_o + lane_addr, c8, o8);
+                if (kFp8) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) o8[k] *= v_scale;
+                }
                 if (c8 * 8 + 8 <= M) {
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) po[k * 128] = __uint_as_float(r[k]);
+                    for (int k = 0; k < 8; ++k) po[k * 128] = o8[k];
                 } else {
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
-                        if (c8 * 8 + k < M) po[k * 128] = __uint_as_float(r[k]);
+                        if (c8 * 8 + k < M) po[k * 128] = o8[k];
                 }
             }
             if (wq == 0) {
 #pragma unroll 1
                 for (int c8 = c_lo; c8 < c_hi; ++c8) {
-                    uint32_t r[8];
-                    tmem_ld_x8(tm_l + c8 * 8, r);     // lane 0: l, lane 1: l_vis
-                    tmem_wait_ld();
+                    float lsum[8];
+                    load_acc8<kFp8>(tm_l, c8, lsum);      // lane 0: l, lane 1: l_vis
                     // lane k takes column k of the chunk: l from lane 0, l_vis from lane 1
                     float lk = 0.f, lvk = 0.f;
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
-                        const float a = __shfl_sync(0xffffffffu, __uint_as_float(r[k]), 0);
-                        const float c = __shfl_sync(0xffffffffu, __uint_as_float(r[k]), 1);
+                        const float a = __shfl_sync(0xffffffffu, lsum[k], 0);
+                        const float c = __shfl_sync(0xffffffffu, lsum[k], 1);
                         if (lane == k) { lk = a; lvk = c; }
                     }
                     if (lane < 8 && c8 * 8 + lane < M)
@@ -804,6 +969,20 @@ bool make_kv_map(CUtensorMap *map, const void *ptr, int Lmax, int BH)
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// [B*Hkv][Lmax][128] E4M3 codes viewed as a 3-D byte tensor; boxes of 128 channels x 128 positions
+bool make_kv_map_fp8(CUtensorMap *map, const void *ptr, int Lmax, int BH)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {128, (cuuint64_t)Lmax, (cuuint64_t)BH};
+    const cuuint64_t strides[2] = {128, (cuuint64_t)Lmax * 128};
+    const cuuint32_t box[3] = {128, 128, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(ptr), dims, strides, box,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // q [B][gamma][Hq][128] bf16 as a 4-D tensor; one box = 64 channels of the G heads of one
 // KV head for all gamma queries: its rows land in shared memory in the order g * G + hg
 bool make_q_map(CUtensorMap *map, const void *ptr, int B, int gamma, int Hq, int G)
@@ -821,20 +1000,25 @@ bool make_q_map(CUtensorMap *map, const void *ptr, int B, int gamma, int Hq, int
 
 constexpr uint32_t kMaxSmem = 232448 - 1024;   // 227 KB less the alignment slack
 
-TcConfig pick_config(int M, int page_slots)
+TcConfig pick_config(int M, int page_slots, bool fp8)
 {
     TcConfig c;
     c.n_pad = (M + 15) & ~15;
     c.page_slots = page_slots;
+    c.slot_bytes = fp8 ? kBoxBytes : kSlotBytes;
     // deepest K/V rings that fit: bytes in flight matter more than a second P buffer,
-    // since the probabilities wait in registers for the buffer anyway
+    // since the probabilities wait in registers for the buffer anyway (an fp8 tile is
+    // half the bytes: twice the slots for the same bytes in flight)
     const int tries[6][3] = {{3, 3, 2}, {3, 3, 1}, {2, 3, 2}, {2, 3, 1}, {2, 2, 2}, {2, 2, 1}};
+    const int tries8[6][3] = {{6, 6, 1}, {5, 6, 1}, {5, 5, 1}, {4, 5, 1}, {4, 4, 1}, {3, 3, 1}};
     for (int t = 0; t < 6; ++t) {
-        c.ks = tries[t][0]; c.vs = tries[t][1]; c.pb = tries[t][2];
+        const int *tr = fp8 ? tries8[t] : tries[t];
+        c.ks = tr[0]; c.vs = tr[1]; c.pb = tr[2];
         if (smem_map(c).total <= kMaxSmem) break;
     }
+    // S^T twice, O^T and the sums: 4 columns per padded row, 6 with an fp8 cache
     int cols = 32;
-    while (cols < 4 * c.n_pad) cols <<= 1;
+    while (cols < (fp8 ? 6 : 4) * c.n_pad) cols <<= 1;
     c.tmem_cols = cols;
     return c;
 }
@@ -843,6 +1027,7 @@ TcConfig pick_config(int M, int page_slots)
 
 bool attn_tc_supported(const AttnParams &p)
 {
+    if (p.fp8 && (p.M > kMaxRowsFp8 || p.page_size > 0 || p.branch_len != p.gamma)) return false;
     return p.D == 128 && p.Lmax >= kTilePos && p.M <= LVSPEC_MAX_ROWS;
 }
 
@@ -853,19 +1038,26 @@ cudaError_t launch_attn_tc(const AttnParams &p, const SeqInfo &seq, cudaStream_t
     const bool paged = p.page_size > 0;
     // paged: one block-table entry per tile of the longest split, rounded up to 4
     const int tiles = (p.Lmax + kTilePos - 1) / kTilePos;
-    P.cfg = pick_config(p.M, paged ? ((tiles + p.n_split - 1) / p.n_split + 4) & ~3 : 0);
-    if (smem_map(P.cfg).total > kMaxSmem) return cudaErrorInvalidConfiguration;
+    const bool fp8 = p.fp8 != 0;
+    P.cfg = pick_config(p.M, paged ? ((tiles + p.n_split - 1) / p.n_split + 4) & ~3 : 0, fp8);
+    if (smem_map(P.cfg).total > kMaxSmem || P.cfg.tmem_cols > 512) return cudaErrorInvalidConfiguration;
     CUtensorMap mk, mv, mq;
     const int map_len = paged ? p.page_size : p.Lmax;
     const int map_rows = paged ? p.n_pages * p.Hkv : p.B * p.Hkv;
-    if (!make_kv_map(&mk, p.k, map_len, map_rows) || !make_kv_map(&mv, p.v, map_len, map_rows) ||
-        !make_q_map(&mq, p.q, p.B, p.gamma, p.Hq, p.G))
+    if (fp8) {
+        if (!make_kv_map_fp8(&mk, p.k, map_len, map_rows) || !make_kv_map_fp8(&mv, p.v, map_len, map_rows))
+            return cudaErrorInvalidValue;
+        mq = mk;     // not used by the kernel
+    } else if (!make_kv_map(&mk, p.k, map_len, map_rows) || !make_kv_map(&mv, p.v, map_len, map_rows) ||
+               !make_q_map(&mq, p.q, p.B, p.gamma, p.Hq, p.G)) {
         return cudaErrorInvalidValue;
+    }
     const size_t smem = smem_map(P.cfg).total + 1024;
     const bool tree = p.branch_len != p.gamma;
-    if (tree && paged) return cudaErrorNotSupported;
-    auto kernel = paged ? attn_tc_kernel<false, true>
-                        : (tree ? attn_tc_kernel<true, false> : attn_tc_kernel<false, false>);
+    if ((tree && paged) || (fp8 && (tree || paged))) return cudaErrorNotSupported;
+    auto kernel = fp8 ? attn_tc_kernel<false, false, true>
+                      : (paged ? attn_tc_kernel<false, true, false>
+                               : (tree ? attn_tc_kernel<true, false, false> : attn_tc_kernel<false, false, false>));
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
