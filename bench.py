@@ -530,6 +530,7 @@ def run_ours(args, cfg):
 
     if not args.no_next_rows and world == 1:
         line["next_rows"] = {"visual_relevance": time_visual_relevance(cfg, ctx, stream, torch, dev, peak, args.top_n),
+                             "fp8_attention": time_fp8_attention(cfg, ctx, stream, vs.ks, vs.vs, vs.qs, torch, dev, peak),
                              "paged_attention": time_paged_attention(cfg, ctx, stream, vs.ks, vs.vs, vs.qs, torch, dev, peak),
                              "several_spans": time_span_layer(cfg, ctx, stream, vs.ks, vs.vs, vs.qs, torch, dev)}
 
@@ -641,6 +642,58 @@ def time_span_layer(cfg, ctx, stream, ks, vs_, qs, torch, dev):
     us_hull = timed(lambda l: ctx.verify_attention(shape, qs[l], ks[l], vs_[l], kv_len, hull, out, mass))
     return {"n_spans": len(frames), "gap_positions": 3 * (len(frames) - 1), "us_per_call": us_spans,
             "us_per_call_one_span": us_hull, "note": "graph replays of four layers' calls"}
+
+
+def time_fp8_attention(cfg, ctx, stream, ks, vs_, qs, torch, dev, peak):
+    """The verify attention on an fp8 (E4M3) cache: the first layers' caches of the step
+    quantised on the device with one scale per KV head (largest magnitude -> 448), in a
+    graph of up to eight layers (each streams its own K/V, more than L2 together).
+    Algorithmic bytes: one byte per cache element, q and out in bf16, the mass."""
+    from paper_2604_05650_b200 import binding
+    B, g, Hq, Hkv, D, L = cfg.batch, cfg.gamma, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.kv_len
+    if D != 128 or g * (Hq // Hkv) > 80:
+        return None
+    n_layers = min(8, len(ks))
+
+    def quantize(t):
+        scale = (t.float().abs().amax(dim=(2, 3)) / 448.0).clamp_min(1e-30)
+        codes = (t.float() / scale[:, :, None, None]).to(torch.float8_e4m3fn).view(torch.uint8)
+        return codes.contiguous(), scale.contiguous()
+
+    k8 = [quantize(ks[l]) for l in range(n_layers)]
+    v8 = [quantize(vs_[l]) for l in range(n_layers)]
+    out = torch.empty((B, g, Hq, D), dtype=torch.bfloat16, device=dev)
+    mass = torch.empty((B, g, Hq), dtype=torch.float32, device=dev)
+    shape = binding.attn_shape(B, g, Hq, Hkv, D, L, 0, 0)
+    kv_len = np.full((B,), L, dtype=np.int32)
+    span = np.tile(np.asarray([cfg.span], dtype=np.int32), (B, 1))
+
+    def layers():
+        for l in range(n_layers):
+            ctx.verify_attention_fp8(shape, qs[l], k8[l][0], v8[l][0], k8[l][1], v8[l][1], kv_len, span, out, mass)
+
+    with torch.cuda.stream(stream):
+        layers()
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            ctx.set_stream(torch.cuda.current_stream().cuda_stream)
+            layers()
+        ctx.set_stream(stream.cuda_stream)
+        for _ in range(3):
+            graph.replay()
+        reps = 20
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            graph.replay()
+        e1.record(stream)
+    stream.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / (reps * n_layers)
+    nbytes = cfg.kv_bytes_per_layer // 2 + 2 * B * Hkv * 4 + 2 * B * g * Hq * D * 2 + B * g * Hq * 4
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return {"us_per_layer": us, "layers_in_graph": n_layers, "bytes_per_layer": nbytes, "achieved_gbs": gbs,
+            "frac_of_peak": gbs / peak, "splits": ctx.attention_splits(shape, L), "cache": "E4M3, one scale per KV head"}
 
 
 def time_paged_attention(cfg, ctx, stream, ks, vs_, qs, torch, dev, peak):
