@@ -107,17 +107,20 @@ int resolve_kernel(const lvspec_attn_shape_t *s)
 }
 
 // KV splits per (sequence, KV head) when the caller leaves the choice to the library.
-// The tensor-core kernel runs one CTA per SM and is bound by HBM once about three
-// quarters of the SMs stream (one SM alone pulls about 60 GB/s).  Splits are whole
+// The tensor-core kernel runs one CTA per SM.  One CTA works through a tile in a time
+// that grows with the query rows it carries (measured: about 2.1 k cycles at 48 padded
+// rows, 2.7 k at 80), so with 40 rows about three quarters of the SMs already stream at
+// the HBM bandwidth, with 80 rows nearly all are needed, and with an fp8 cache (half the
+// bytes per tile for the same work) the device never gets there.  Splits are whole
 // 128-position tiles, so a split count that does not divide the tile count leaves a last
 // round in which only the CTAs with one tile more are at work, far below the device's
-// bandwidth: 16 splits of 16 tiles beat 18 splits of 14 or 15 on eight heads of 256 tiles.
-// The count is therefore chosen by a small model of the stream, in units of the time the
-// whole device takes for one tile: the even rounds at the bandwidth their CTA count
-// reaches, the uneven last round at the bandwidth of its few CTAs, and a charge per CTA
-// for writing its partial and merging it.  A pure function of the shape: results stay
-// reproducible from run to run.
-int choose_splits(const lvspec_ctx *ctx, const lvspec_attn_shape_t *s, int max_kv_len)
+// bandwidth: with 40 rows, 16 splits of 16 tiles beat 18 splits of 14 or 15 on eight
+// heads of 256 tiles.  The count is therefore chosen by a small model of the stream, in
+// units of the time the whole device takes for one tile: the even rounds at the bandwidth
+// their CTA count reaches, the uneven last round at the bandwidth of its few CTAs, and a
+// charge per CTA for writing its partial and merging it.  A pure function of the shape:
+// results stay reproducible from run to run.
+int choose_splits(const lvspec_ctx *ctx, const lvspec_attn_shape_t *s, int max_kv_len, bool fp8 = false)
 {
     const int tiles = (max_kv_len + 127) / 128;           // splits never go below 128 positions
     const int units = s->batch * s->n_kv_heads;
@@ -132,7 +135,12 @@ int choose_splits(const lvspec_ctx *ctx, const lvspec_attn_shape_t *s, int max_k
     if (most < 1) most = 1;
     if (most > tiles) most = tiles;
     if (most > 256) most = 256;
-    const double saturating = 0.73 * ctx->n_sm;            // CTAs that reach the HBM bandwidth
+    // CTAs that reach the HBM bandwidth
+    const int n_pad = (s->gamma * (s->n_q_heads / s->n_kv_heads) + 15) & ~15;
+    double share = 0.73 * (1100.0 + 20.0 * n_pad) / (1100.0 + 20.0 * 48);
+    if (share < 0.6) share = 0.6;
+    if (fp8) share *= 2.3;
+    const double saturating = share * ctx->n_sm;
     auto rate = [&](double ctas) { return ctas >= saturating ? 1.0 : ctas / saturating; };
     int best = most;
     double best_cost = 0.0;
@@ -248,7 +256,7 @@ lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, con
     p.Lmax = s->kv_capacity;
     p.G = p.Hq / p.Hkv;
     p.M = p.gamma * p.G;
-    p.n_split = s->n_split > 0 ? s->n_split : choose_splits(ctx, s, max_len);
+    p.n_split = s->n_split > 0 ? s->n_split : choose_splits(ctx, s, max_len, fp8 != nullptr);
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)p.D));
     p.pdl = ctx->pdl ? 1 : 0;
     p.branch_len = branch_len > 0 ? branch_len : p.gamma;
@@ -512,7 +520,13 @@ size_t lvspec_attention_workspace_bytes(const lvspec_ctx_t *ctx, const lvspec_at
     if (!ctx || !shape || shape->batch < 1 || shape->n_kv_heads < 1 || shape->gamma < 1 ||
         shape->n_q_heads < shape->n_kv_heads || shape->head_dim < 1 || max_kv_len < 1 || shape->n_split < 0)
         return 0;
-    const int n_split = shape->n_split > 0 ? shape->n_split : choose_splits(ctx, shape, max_kv_len);
+    // the library's own choice differs between the bf16 and the fp8 cache: the larger of the two
+    int n_split = shape->n_split;
+    if (n_split == 0) {
+        n_split = choose_splits(ctx, shape, max_kv_len);
+        const int n8 = choose_splits(ctx, shape, max_kv_len, true);
+        if (n8 > n_split) n_split = n8;
+    }
     // the call with several spans never runs the tensor-core kernel on a single split
     const int n_eff = n_split < 2 ? 2 : n_split;
     const int M = shape->gamma * (shape->n_q_heads / shape->n_kv_heads);

@@ -282,6 +282,13 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
+// largest value over the warp's 32 lanes (one instruction on sm_100a; NaN inputs are passed over)
+__device__ __forceinline__ float warp_max_f32(float x)
+{
+    float r;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(x));
+    return r;
+}
 // two fp32 -> packed E4M3 pair (lo in the low byte), round to nearest even, saturating
 __device__ __forceinline__ uint32_t pack_e4m3x2(float lo, float hi)
 {

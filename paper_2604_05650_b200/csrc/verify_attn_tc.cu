@@ -751,9 +751,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                         float s2 = __uint_as_float(r[k]) * scale;
                         if (tail && (kTree ? !column_sees(vis_s[c8 * 8 + k], gmin) : (c8 * 8 + k) / G < gmin))
                             s2 = -INFINITY;
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1)
-                            s2 = fmaxf(s2, __shfl_xor_sync(0xffffffffu, s2, o));
+                        s2 = warp_max_f32(s2);
                         if (lane == 0) tmx_s[wq * NP + c8 * 8 + k] = s2;
                     }
                 }
@@ -1010,7 +1008,7 @@ TcConfig pick_config(int M, int page_slots, bool fp8)
     // since the probabilities wait in registers for the buffer anyway (an fp8 tile is
     // half the bytes: twice the slots for the same bytes in flight)
     const int tries[6][3] = {{3, 3, 2}, {3, 3, 1}, {2, 3, 2}, {2, 3, 1}, {2, 2, 2}, {2, 2, 1}};
-    const int tries8[6][3] = {{6, 6, 1}, {5, 6, 1}, {5, 5, 1}, {4, 5, 1}, {4, 4, 1}, {3, 3, 1}};
+    const int tries8[6][3] = {{5, 6, 2}, {5, 5, 2}, {4, 5, 2}, {4, 4, 2}, {4, 4, 1}, {3, 3, 1}};
     for (int t = 0; t < 6; ++t) {
         const int *tr = fp8 ? tries8[t] : tries[t];
         c.ks = tr[0]; c.vs = tr[1]; c.pb = tr[2];
