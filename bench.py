@@ -597,7 +597,7 @@ def time_visual_relevance(cfg, ctx, stream, torch, dev, peak, top_n=10):
     nbytes = B * lv * d * 2 + B * lv * 4
     gbs = nbytes / (us * 1e-6) / 1e9
     return {"us_per_call": us, "n_visual": lv, "dim": d, "top_n": top_n, "bytes_per_call": nbytes,
-            "achieved_gbs": gbs, "frac_of_peak": gbs / peak, "launches_per_call": 3}
+            "achieved_gbs": gbs, "frac_of_peak": gbs / peak, "launches_per_call": 2}
 
 
 def time_span_layer(cfg, ctx, stream, ks, vs_, qs, torch, dev):

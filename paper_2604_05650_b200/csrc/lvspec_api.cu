@@ -19,6 +19,7 @@ struct lvspec_ctx {
     cudaStream_t stream = nullptr;
     uint32_t *status = nullptr;       // device status word
     uint32_t *counters = nullptr;     // [LVSPEC_MAX_BATCH] tickets of the acceptance kernel
+    uint32_t *rel_counters = nullptr; // [LVSPEC_MAX_BATCH * LVSPEC_MAX_GAMMA] candidate counts of the relevance score
     void *scratch = nullptr;          // split partials / argmax partials
     size_t scratch_bytes = 0;
     void *staging = nullptr;          // device copies for the *_host calls
@@ -426,7 +427,7 @@ lvspec_status_t lvspec_create(lvspec_ctx_t **out, int device)
     }
     ctx->n_sm = prop.multiProcessorCount;
     if (const char *e = std::getenv("LVSPEC_NO_PDL")) ctx->pdl = !(e[0] && e[0] != '0');
-    const size_t small = sizeof(uint32_t) * (1 + LVSPEC_MAX_BATCH);
+    const size_t small = sizeof(uint32_t) * (1 + LVSPEC_MAX_BATCH + LVSPEC_MAX_BATCH * LVSPEC_MAX_GAMMA);
     if ((e = cudaMalloc(reinterpret_cast<void **>(&ctx->status), small)) != cudaSuccess ||
         (e = cudaMemset(ctx->status, 0, small)) != cudaSuccess) {
         g_create_error = std::string("status allocation: ") + cudaGetErrorString(e);
@@ -436,6 +437,7 @@ lvspec_status_t lvspec_create(lvspec_ctx_t **out, int device)
         return LVSPEC_ERR_WORKSPACE;
     }
     ctx->counters = ctx->status + 1;
+    ctx->rel_counters = ctx->counters + LVSPEC_MAX_BATCH;
     lvspec_status_t st = ensure(ctx, &ctx->scratch, &ctx->scratch_bytes, size_t(8) << 20, true);
     if (st != LVSPEC_OK) {
         g_create_error = ctx->error;
@@ -857,6 +859,7 @@ lvspec_status_t lvspec_visual_relevance(lvspec_ctx_t *ctx, int32_t batch, int32_
     p.v_inv_norm = visual_inv_norm;
     p.cos_t = static_cast<float *>(ctx->scratch);
     p.relevance = relevance;
+    p.counters = ctx->rel_counters;
     p.status = ctx->status;
     p.B = batch;
     p.K = gamma;

@@ -107,8 +107,9 @@ struct RelevanceParams {
     const uint16_t *h_draft;    // [B, K, d] bf16
     const uint16_t *h_visual;   // [B, lv, d] bf16
     const float *v_inv_norm;    // [B, lv]
-    float *cos_t;               // scratch [B, K, lv_pad]: cosines, one contiguous row per draft token
+    float *cos_t;               // scratch [B, K, lv_pad]: Top-N candidates or all cosines, one row per draft token
     float *relevance;           // [B, K]
+    uint32_t *counters;         // [B, K] candidates appended so far; zero between calls
     uint32_t *status;
     int32_t B, K, lv, d, top_n;
     int32_t lv_pad;             // lv rounded up to a multiple of 4

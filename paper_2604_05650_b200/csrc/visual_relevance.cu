@@ -2,17 +2,22 @@
 // token the mean of the N largest cosine similarities between its final-layer
 // hidden state and the visual tokens' final-layer hidden states.
 //
-// Three kernels per call:
-//   draft_prep_kernel   copies H_D into a row-padded scratch tile (rows padded to
-//                       a multiple of 16 with zeros) and takes its reciprocal norms
+// Two kernels per call:
 //   cos_tc_kernel       streams H_V once (the HBM-bound part): every CTA takes an
 //                       equal share of the visual rows, in chunks of up to 256
 //                       rows = two row blocks with one accumulator each;
 //                       S[row, k] = H_V[row, :] . H_D[k, :] on the tensor core
-//                       (tcgen05, MMA M = 128 rows, N = padded K, the hidden
-//                       dimension in TMA stages of 64 channels), then
-//                       cosine = S * inv_norm_v[row] * inv_norm_d[k] to scratch
-//   topn_mean_kernel    exact Top-N mean per draft token by radix selection
+//                       (tcgen05, MMA M = 128 rows, N = K padded to 16 by the TMA
+//                       unit's zero fill, the hidden dimension in TMA stages of 64
+//                       channels); its otherwise idle epilogue warps take H_D's
+//                       reciprocal norms meanwhile; then
+//                       cosine = S * inv_norm_v[row] * inv_norm_d[k].
+//                       N <= 32: every warp keeps, per draft token, only the N largest
+//                       cosines of its 32 rows (they hold every value the exact Top-N
+//                       can contain) and appends them to the token's candidate list;
+//                       N > 32: all cosines go to scratch.
+//   topn_mean_kernel    exact Top-N mean per draft token over the candidates (or
+//                       all cosines), summed in descending order of value
 // The reciprocal norms of H_V's rows come from row_inv_norms_kernel, run once
 // after prefill.
 #include <cuda.h>
@@ -56,77 +61,55 @@ row_inv_norms_kernel(const uint16_t *x, long long rows, int dim, float *out)
     if (lane == 0) out[r] = acc > 0.f ? 1.f / sqrtf(acc) : 0.f;
 }
 
-// H_D [B, K, d] -> hd_pad [B, NP, d] (rows >= K zero) and dinv [B, NP]; one CTA per padded row
-constexpr int kPrepThreads = 256;
-__global__ void __launch_bounds__(kPrepThreads)
-draft_prep_kernel(const uint16_t *hd, int B, int K, int NP, int dim, uint16_t *hd_pad, float *dinv)
-{
-    __shared__ float part[kPrepThreads / 32];
-    // the streaming kernel may be scheduled at once (it sets itself up, then waits for
-    // this grid); this grid waits for whatever ran before it in the stream
-    grid_launch_dependents();
-    grid_dependency_wait();
-    const int r = blockIdx.x;                       // padded row index over B * NP
-    const int b = r / NP, k = r - b * NP;
-    uint4 *dst = reinterpret_cast<uint4 *>(hd_pad + (size_t)r * dim);
-    if (k >= K) {
-        for (int i = threadIdx.x; i < dim / 8; i += kPrepThreads) dst[i] = make_uint4(0, 0, 0, 0);
-        if (threadIdx.x == 0) dinv[r] = 0.f;
-        return;
-    }
-    const uint4 *src = reinterpret_cast<const uint4 *>(hd + ((size_t)b * K + k) * dim);
-    float acc = 0.f;
-    for (int i = threadIdx.x; i < dim / 8; i += kPrepThreads) {
-        const uint4 w = __ldg(src + i);
-        dst[i] = w;
-        acc = sumsq_bf16x8(w, acc);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = acc;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float t = 0.f;
-        for (int w = 0; w < kPrepThreads / 32; ++w) t += part[w];
-        dinv[r] = t > 0.f ? 1.f / sqrtf(t) : 0.f;
-    }
-}
-
 // ------------------------------------------------------------- cosine kernel
 constexpr int kCosThreads = 192;            // warp 0 producer, warp 1 MMA, warps 2-5 epilogue
 constexpr uint32_t kGroupBytes = 2048;      // 16 rows x 64 channels bf16
 constexpr uint32_t kBlockBytes = 8 * kGroupBytes;    // one row block: 128 rows
-constexpr int kChunkGroups = 16;            // groups of 16 rows per chunk
+constexpr int kChunkGroups = 16;            // most groups of 16 rows per chunk
 constexpr int kMaxStages = 24;
 constexpr uint32_t kBarBytes = 1024;        // barriers and the TMEM slot, ahead of the stages
 
+constexpr int kTopFused = 32;               // Top-N up to this is selected per warp in the cosine kernel
+constexpr uint32_t kDinvOffset = 704;       // reciprocal norms of H_D's rows, inside the barrier block
+
 struct CosParams {
     RelevanceParams r;
-    const float *dinv;      // [B, NP]
     int NP;                 // K padded to a multiple of 16 (MMA N)
     int smem_bytes;         // dynamic shared memory of the launch (after 1024-byte alignment)
     int tmem_cols;
     int tail_a, tail_b;     // row-group counts that have a one-box tensor map of their own (0 = none)
     int n_grp;              // groups of 16 rows per batch element
     int total_groups;       // B * n_grp
+    int chunk_groups;       // groups of 16 rows per chunk (<= kChunkGroups)
 };
 
 // The chunks (up to 16 groups of 16 rows of one batch element) of one CTA's share
 // of the row groups; producer, MMA issuer and epilogue walk them in step.
 struct ChunkWalk {
-    int gg, end, n_grp;
+    int gg, end, n_grp, chunk_groups;
     int b, row0, n_groups;   // the current chunk
     __device__ bool next()
     {
         if (gg >= end) return false;
         b = gg / n_grp;
         const int g0 = gg - b * n_grp;
-        n_groups = min(kChunkGroups, min(n_grp - g0, end - gg));
+        n_groups = min(chunk_groups, min(n_grp - g0, end - gg));
         row0 = g0 * 16;
         gg += n_groups;
         return true;
     }
 };
+
+// order-preserving map float -> unsigned (larger float, larger key)
+__device__ __forceinline__ uint32_t float_key(float v)
+{
+    const uint32_t u = __float_as_uint(v);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_float(uint32_t k)
+{
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
 
 __device__ __forceinline__ bool wait_teardown(uint32_t bar, uint32_t parity)
 {
@@ -154,11 +137,12 @@ cos_tc_kernel(const CosParams P, const __grid_constant__ CUtensorMap tmap_v,
         walk.gg = c * per + min(c, rem);
         walk.end = walk.gg + per + (c < rem ? 1 : 0);
         walk.n_grp = P.n_grp;
+        walk.chunk_groups = P.chunk_groups;
     }
     // A stage holds 64 channels of the tallest chunk this CTA can meet (row block 0,
     // then row block 1, then the draft tile); the fewer rows, the more stages fit,
     // and bytes in flight, not stages, are what covers the memory latency.
-    const int cap = max(1, min(kChunkGroups, walk.end - walk.gg));
+    const int cap = max(1, min(P.chunk_groups, walk.end - walk.gg));
     const uint32_t d_off = cap <= 8 ? (uint32_t)cap * kGroupBytes : kBlockBytes + (uint32_t)(cap - 8) * kGroupBytes;
     const uint32_t stage_bytes = (d_off + (uint32_t)NP * 128u + 1023u) & ~1023u;
     // An MMA always reads whole row blocks of 128 rows (rows a chunk does not have are
@@ -299,28 +283,93 @@ cos_tc_kernel(const CosParams P, const __grid_constant__ CUtensorMap tmap_v,
         const int wq = warp & 3;
         const int row = wq * 32 + lane;                    // TMEM lane = row inside the chunk
         const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
-        int chunk = 0;
+        float *dinv_s = reinterpret_cast<float *>(gbase + kDinvOffset);
+        const bool fused = p.top_n <= kTopFused;
+        const int n_it = min(p.top_n, 32);
+        int chunk = 0, cur_b = -1;
         while (walk.next()) {
+            if (walk.b != cur_b) {
+                // reciprocal norms of this batch element's draft rows: a warp per row,
+                // while the rows of H_V stream in (fixed summation order)
+                if (cur_b >= 0) asm volatile("bar.sync 1, 128;" ::: "memory");   // the old ones are no longer read
+                cur_b = walk.b;
+                for (int k = wq; k < NP; k += 4) {
+                    float acc = 0.f;
+                    if (k < p.K) {
+                        const uint4 *src = reinterpret_cast<const uint4 *>(p.h_draft + ((size_t)cur_b * p.K + k) * p.d);
+                        for (int i = lane; i < p.d / 8; i += 32) acc = sumsq_bf16x8(__ldg(src + i), acc);
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+                    }
+                    if (lane == 0) dinv_s[k] = acc > 0.f ? 1.f / sqrtf(acc) : 0.f;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+            }
             const int buf = chunk & 1;
             mbar_wait(acc_full(buf), (chunk >> 1) & 1, abort_flag);
             tc_fence_after();
-            const float *dinv = P.dinv + (size_t)walk.b * NP;
             const int n_blocks = walk.n_groups > 8 ? 2 : 1;
             for (int blk = 0; blk < n_blocks; ++blk) {
                 const int rc = blk * 128 + row;                // row inside the chunk
                 const int j = walk.row0 + rc;                  // visual row of this thread
                 const bool valid = rc < walk.n_groups * 16 && j < p.lv;
                 const float vin = valid ? __ldg(p.v_inv_norm + (size_t)walk.b * p.lv + j) : 0.f;
-                float *dst = p.cos_t + (size_t)walk.b * p.K * p.lv_pad + j;
-                for (int c8 = 0; c8 < NP / 8; ++c8) {
+                float *dst = p.cos_t + (size_t)walk.b * p.K * p.lv_pad;
+                if (fused && __ballot_sync(0xffffffffu, valid) == 0u) continue;     // no row of this warp in the chunk
+                for (int c8 = 0; c8 < NP / 8 && c8 * 8 < p.K; ++c8) {
                     uint32_t r[8];
                     tmem_ld_x8(tmem_base + (buf * 2 + blk) * NP + lane_addr + c8 * 8, r);
                     tmem_wait_ld();
+                    if (!fused) {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            const int kk = c8 * 8 + k;
+                            if (valid && kk < p.K)
+                                dst[(size_t)kk * p.lv_pad + j] = __uint_as_float(r[k]) * vin * dinv_s[kk];
+                        }
+                        continue;
+                    }
+                    // the N largest of this warp's 32 rows, per draft token: the warp sorts
+                    // the 32 keys of a column with shuffles (descending; the eight columns
+                    // side by side), lane t then holds the t-th largest.  Key 0 = no value.
+                    uint32_t top[8];
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
                         const int kk = c8 * 8 + k;
-                        if (valid && kk < p.K)
-                            dst[(size_t)kk * p.lv_pad] = __uint_as_float(r[k]) * vin * __ldg(dinv + kk);
+                        top[k] = (valid && kk < p.K) ? float_key(__uint_as_float(r[k]) * vin * dinv_s[kk]) : 0u;
+                    }
+#pragma unroll
+                    for (int size = 2; size <= 32; size <<= 1) {
+#pragma unroll
+                        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+                            const bool upper = (lane & stride) != 0;          // holds the second of the pair
+                            const bool descending = (lane & size) == 0;
+                            const bool take_max = (upper != descending);      // first of a descending pair keeps the max
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const uint32_t y = __shfl_xor_sync(0xffffffffu, top[k], stride);
+                                top[k] = take_max ? max(top[k], y) : min(top[k], y);
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        if (lane >= n_it) top[k] = 0u;
+                    // lane k reserves the places of column k: the eight requests travel together
+                    uint32_t my_cnt = 0u;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const uint32_t cnt = __popc(__ballot_sync(0xffffffffu, top[k] != 0u));
+                        if (lane == k) my_cnt = cnt;
+                    }
+                    uint32_t my_off = 0u;
+                    if (lane < 8 && c8 * 8 + lane < p.K && my_cnt > 0u)
+                        my_off = atomicAdd(p.counters + (size_t)walk.b * p.K + c8 * 8 + lane, my_cnt);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const int kk = c8 * 8 + k;
+                        const uint32_t off = __shfl_sync(0xffffffffu, my_off, k);
+                        if (kk < p.K && top[k] != 0u) dst[(size_t)kk * p.lv_pad + off + lane] = key_float(top[k]);
                     }
                 }
             }
@@ -350,17 +399,6 @@ cos_tc_kernel(const CosParams P, const __grid_constant__ CUtensorMap tmap_v,
 
 // ------------------------------------------------------------- Top-N mean
 constexpr int kTopThreads = 1024;
-
-// order-preserving map float -> unsigned (larger float, larger key)
-__device__ __forceinline__ uint32_t float_key(float v)
-{
-    const uint32_t u = __float_as_uint(v);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-__device__ __forceinline__ float key_float(uint32_t k)
-{
-    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
-}
 
 constexpr int kTopPerThread = 32;      // fast path: lv <= 32 * 1024
 constexpr int kTopCandidates = 2048;
@@ -399,11 +437,28 @@ __global__ void __launch_bounds__(kTopThreads) topn_mean_kernel(const RelevanceP
     __shared__ uint32_t hist[256];
     __shared__ uint32_t sel_prefix, sel_need, n_cand;
     __shared__ float warp_sum[kTopThreads / 32];
+    __shared__ int n_values;
     const int k = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
     const float *row = p.cos_t + ((size_t)b * p.K + k) * p.lv_pad;
-    const int lv = p.lv;
-    const uint32_t n = (uint32_t)min(p.top_n, lv);
+    // with N <= kTopFused the row holds the candidates the cosine kernel appended (at
+    // least min(N, lv) of them, every value of the exact Top-N among them) and the
+    // counter says how many; the counter goes back to zero for the next call
+    if (tid == 0) {
+        n_values = p.lv;
+        if (p.top_n <= kTopFused) {
+            uint32_t *cnt = p.counters + (size_t)b * p.K + k;
+            n_values = (int)min(__ldcg(cnt), (uint32_t)p.lv);
+            *cnt = 0u;
+        }
+    }
+    __syncthreads();
+    const int lv = n_values;
+    const uint32_t n = (uint32_t)min(p.top_n, p.lv);
     float *out = p.relevance + (size_t)b * p.K + k;
+    if ((uint32_t)lv < n) {       // cannot happen unless the cosine kernel gave up on a wait
+        if (tid == 0) *out = __int_as_float(0x7fc00000);
+        return;
+    }
 
     if (lv <= kTopPerThread * kTopThreads && n <= (uint32_t)kTopThreads) {
         uint32_t mine[kTopPerThread];
@@ -558,46 +613,24 @@ cudaError_t launch_row_inv_norms(const uint16_t *x, long long rows, int dim, flo
     return cudaGetLastError();
 }
 
-// Scratch layout behind p.cos_t: cosines [B, K, lv_pad] fp32, then the padded draft
-// tile [B, NP, d] bf16 (1024-byte aligned), then its reciprocal norms [B, NP].
+// Scratch behind p.cos_t: per (sequence, draft token) a row of lv_pad fp32 values (the
+// Top-N candidates, or all cosines when N is large).
 size_t relevance_scratch_bytes(int B, int K, int lv, int d)
 {
-    const int NP = (K + 15) & ~15;
+    (void)d;
     const int lv_pad = (lv + 3) & ~3;
-    size_t o = (size_t)B * K * lv_pad * sizeof(float);
-    o = (o + 1023) & ~size_t(1023);
-    o += (size_t)B * NP * d * 2;
-    o = (o + 1023) & ~size_t(1023);
-    o += (size_t)B * NP * sizeof(float);
-    return o;
+    return (size_t)B * K * lv_pad * sizeof(float);
 }
 
 cudaError_t launch_visual_relevance(const RelevanceParams &p, cudaStream_t stream, int *launches)
 {
     const int NP = (p.K + 15) & ~15;
-    size_t o = (size_t)p.B * p.K * p.lv_pad * sizeof(float);
-    o = (o + 1023) & ~size_t(1023);
-    uint16_t *hd_pad = reinterpret_cast<uint16_t *>(reinterpret_cast<char *>(p.cos_t) + o);
-    o += (size_t)p.B * NP * p.d * 2;
-    o = (o + 1023) & ~size_t(1023);
-    float *dinv = reinterpret_cast<float *>(reinterpret_cast<char *>(p.cos_t) + o);
-
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cudaLaunchConfig_t cfg0 = {};
-    cfg0.gridDim = dim3((unsigned)(p.B * NP), 1, 1);
-    cfg0.blockDim = dim3(kPrepThreads, 1, 1);
-    cfg0.stream = stream;
-    cfg0.attrs = attr;
-    cfg0.numAttrs = 1;
-    cudaError_t err = cudaLaunchKernelEx(&cfg0, draft_prep_kernel, p.h_draft, p.B, p.K, NP, p.d, hd_pad, dinv);
-    ++*launches;
-    if (err != cudaSuccess) return err;
 
     CosParams P;
     P.r = p;
-    P.dinv = dinv;
     P.NP = NP;
     P.smem_bytes = 232448 - 1024;      // everything an SM offers, less the alignment slack
     int cols = 32;
@@ -606,8 +639,12 @@ cudaError_t launch_visual_relevance(const RelevanceParams &p, cudaStream_t strea
     P.n_grp = (p.lv + 15) / 16;
     P.total_groups = p.B * P.n_grp;
     // The shares are `per` or `per + 1` groups; what a share leaves after its full chunks
-    // and its full row block is the tail that gets a map of its own.
+    // and its full row block is the tail that gets a map of its own.  (Chunks as tall as
+    // possible: every stage of a chunk costs the producer the same two or three TMA
+    // requests whatever its height; shares cut into three chunks of 64 rows, so that
+    // epilogues could run beside the stream, took twice the time.)
     const int n_cta = P.total_groups < p.n_sm ? P.total_groups : p.n_sm;
+    P.chunk_groups = kChunkGroups;
     auto tail_of = [](int groups) {
         const int t = groups % kChunkGroups;
         return t > 8 ? t - 8 : t;       // 0..8 groups
@@ -622,10 +659,11 @@ cudaError_t launch_visual_relevance(const RelevanceParams &p, cudaStream_t strea
         !make_rows_map(&mv128, p.h_visual, p.d, p.lv, p.B, p.lv >= 128 ? 128 : 16) ||
         !make_rows_map(&mva, p.h_visual, p.d, p.lv, p.B, P.tail_a > 0 ? P.tail_a * 16 : 16) ||
         !make_rows_map(&mvb, p.h_visual, p.d, p.lv, p.B, P.tail_b > 0 ? P.tail_b * 16 : 16) ||
-        !make_rows_map(&md, hd_pad, p.d, NP, p.B, NP))
+        // the draft rows as they are: the box is NP rows high, the rows beyond K read as zeros
+        !make_rows_map(&md, p.h_draft, p.d, p.K, p.B, NP))
         return cudaErrorInvalidValue;
     const size_t smem = (size_t)P.smem_bytes + 1024;
-    err = cudaFuncSetAttribute(cos_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t err = cudaFuncSetAttribute(cos_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)n_cta, 1, 1);
