@@ -208,6 +208,29 @@ lvspec_status_t lvspec_verify_attention(lvspec_ctx_t *ctx, const lvspec_attn_sha
                                         const int32_t *kv_len, const int32_t *visual_span,
                                         void *out, float *visual_mass);
 
+/* lvspec_verify_attention on a cache with the caller's own layout: any layout in which
+ * the head_dim channels of one (sequence, KV head, position) are contiguous.  Element
+ * (b, h, j, c) of the K cache sits at k_cache + b * k_strides->batch + h * k_strides->head
+ * + j * k_strides->position + c (in bf16 elements), V likewise with v_strides.  The dense
+ * [B, Hkv, Lmax, D] layout of lvspec_verify_attention is {Hkv * Lmax * D, Lmax * D, D};
+ * a position-major cache [B, Lmax, Hkv, D] is {Lmax * Hkv * D, D, Hkv * D}; K and V
+ * interleaved in one buffer [B, Hkv, Lmax, 2, D] is {2 * Hkv * Lmax * D, 2 * Lmax * D, 2 * D}
+ * for both, with v_cache = k_cache + D.  Strides must be positive multiples of 8 elements
+ * (16 bytes), the position stride at least D.  The same operation, arithmetic and
+ * results as lvspec_verify_attention (Eq. 1); the tensor-core kernel reads the layout
+ * through its TMA descriptors, the plain kernel through the same strides. */
+typedef struct {
+    int64_t batch;    /* elements between sequences */
+    int64_t head;     /* elements between KV heads */
+    int64_t position; /* elements between cache positions */
+} lvspec_kv_strides_t;
+lvspec_status_t lvspec_verify_attention_strided(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                                const lvspec_kv_strides_t *k_strides,
+                                                const lvspec_kv_strides_t *v_strides, const void *q,
+                                                const void *k_cache, const void *v_cache,
+                                                const int32_t *kv_len, const int32_t *visual_span,
+                                                void *out, float *visual_mass);
+
 /* Draft-token trees (App. "Exploration on Draft Token Trees": a static tree of
  * branches with K draft tokens each; every branch is verified loosely on its
  * own and the branch with the longest accepted length is kept).

@@ -34,7 +34,7 @@ EXPORTS = (
     "lvspec_verify_attention_spans", "lvspec_last_device_status",
     "lvspec_attention_workspace_bytes", "lvspec_accept_workspace_bytes",
     "lvspec_relevance_workspace_bytes", "lvspec_workspace_capacity", "lvspec_reserve",
-    "lvspec_verify_attention_fp8",
+    "lvspec_verify_attention_fp8", "lvspec_verify_attention_strided",
 )
 
 
@@ -42,6 +42,10 @@ class AttnShape(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("batch", "gamma", "n_q_heads", "n_kv_heads", "head_dim", "kv_capacity",
                  "n_split", "kernel")]
+
+
+class KvStrides(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int64), ("head", ctypes.c_int64), ("position", ctypes.c_int64)]
 
 
 class Thresholds(ctypes.Structure):
@@ -97,6 +101,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lvspec_verify_attention.argtypes = [vp, S, vp, vp, vp, vp, vp, vp, vp]
     lib.lvspec_verify_attention_host.argtypes = [vp, S, vp, vp, vp, vp, vp, vp, vp]
     lib.lvspec_verify_attention_fp8.argtypes = [vp, S, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    KS = ctypes.POINTER(KvStrides)
+    lib.lvspec_verify_attention_strided.argtypes = [vp, S, KS, KS, vp, vp, vp, vp, vp, vp, vp]
     lib.lvspec_loose_accept.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp]
     lib.lvspec_loose_accept_ex.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp, vp, vp]
     lib.lvspec_loose_accept_host.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, T, i32, vp]
@@ -213,6 +219,17 @@ class Context:
         self._check(self._lib.lvspec_verify_attention(
             self._h, ctypes.byref(shape), _addr(q), _addr(k_cache), _addr(v_cache),
             kv_len.ctypes.data, span.ctypes.data, _addr(out), _addr(visual_mass)))
+
+    def verify_attention_strided(self, shape: AttnShape, k_strides, v_strides, q, k_cache, v_cache, kv_len,
+                                 visual_span, out, visual_mass) -> None:
+        """k_strides / v_strides: (batch, head, position) strides in elements."""
+        kv_len, span = _i32(kv_len), _i32(visual_span)
+        if shape.batch >= 1 and (kv_len.size != shape.batch or span.size != 2 * shape.batch):
+            raise ValueError("kv_len needs B entries and visual_span B pairs")
+        ks, vs = KvStrides(*[int(x) for x in k_strides]), KvStrides(*[int(x) for x in v_strides])
+        self._check(self._lib.lvspec_verify_attention_strided(
+            self._h, ctypes.byref(shape), ctypes.byref(ks), ctypes.byref(vs), _addr(q), _addr(k_cache),
+            _addr(v_cache), kv_len.ctypes.data, span.ctypes.data, _addr(out), _addr(visual_mass)))
 
     def verify_attention_fp8(self, shape: AttnShape, q, k_cache, v_cache, k_scale, v_scale, kv_len,
                              visual_span, out, visual_mass) -> None:

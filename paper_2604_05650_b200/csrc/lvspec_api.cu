@@ -239,7 +239,9 @@ struct Fp8Cache {            // E4M3 codes with one scale per (sequence, KV head
 lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, const SeqInfo &seq,
                               int max_len, const void *q, const void *k, const void *v, void *out,
                               float *mass, int branch_len = 0, const PagedCache *paged = nullptr,
-                              float **lse2 = nullptr, const Fp8Cache *fp8 = nullptr)
+                              float **lse2 = nullptr, const Fp8Cache *fp8 = nullptr,
+                              const lvspec_kv_strides_t *k_strides = nullptr,
+                              const lvspec_kv_strides_t *v_strides = nullptr)
 {
     AttnParams p;
     std::memset(&p, 0, sizeof p);
@@ -266,12 +268,20 @@ lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, con
         p.k_scale = fp8->k_scale;
         p.v_scale = fp8->v_scale;
     }
+    // cache strides: dense [B, Hkv, Lmax, D] unless the caller gave its own
+    p.k_sp = p.v_sp = p.D;
+    p.k_sh = p.v_sh = (int64_t)p.Lmax * p.D;
+    p.k_sb = p.v_sb = (int64_t)p.Hkv * p.Lmax * p.D;
     if (paged) {
         p.block_table = paged->block_table;
         p.page_size = paged->page_size;
         p.pages_per_seq = paged->pages_per_seq;
         p.n_pages = paged->n_pages;
+        p.k_sh = p.v_sh = (int64_t)p.page_size * p.D;          // pools [n_pages, Hkv, page_size, D]
+        p.k_sb = p.v_sb = (int64_t)p.Hkv * p.page_size * p.D;
     }
+    if (k_strides) { p.k_sb = k_strides->batch; p.k_sh = k_strides->head; p.k_sp = k_strides->position; }
+    if (v_strides) { p.v_sb = v_strides->batch; p.v_sh = v_strides->head; p.v_sp = v_strides->position; }
 
     const size_t o_bytes = part_o_elems(p) * sizeof(float);
     const size_t st_bytes = part_stat_elems(p) * sizeof(float);
@@ -573,6 +583,33 @@ lvspec_status_t lvspec_verify_attention(lvspec_ctx_t *ctx, const lvspec_attn_sha
     cudaError_t e = cudaSetDevice(ctx->device);
     if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
     return run_attention(ctx, shape, seq, max_len, q, k_cache, v_cache, out, visual_mass);
+}
+
+lvspec_status_t lvspec_verify_attention_strided(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                                const lvspec_kv_strides_t *k_strides,
+                                                const lvspec_kv_strides_t *v_strides, const void *q,
+                                                const void *k_cache, const void *v_cache,
+                                                const int32_t *kv_len, const int32_t *visual_span,
+                                                void *out, float *visual_mass)
+{
+    SeqInfo seq;
+    int max_len = 0;
+    lvspec_status_t st = check_attention(ctx, shape, q, k_cache, v_cache, kv_len, visual_span, out,
+                                         visual_mass, true, &seq, &max_len);
+    if (st != LVSPEC_OK) return st;
+    if (!k_strides || !v_strides) return fail(ctx, LVSPEC_ERR_INVALID_ARG, "null argument");
+    for (const lvspec_kv_strides_t *t : {k_strides, v_strides}) {
+        // a position's channels must not overlap the next position's; 16-byte granularity
+        if (t->position < shape->head_dim || t->head < 1 || t->batch < 1 || (t->position & 7) || (t->head & 7) ||
+            (t->batch & 7) || t->position >= (int64_t(1) << 38) || t->head >= (int64_t(1) << 38) ||
+            t->batch >= (int64_t(1) << 38))
+            return fail(ctx, LVSPEC_ERR_INVALID_ARG,
+                        "cache strides must be positive multiples of 8 elements, the position stride at least head_dim");
+    }
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaSetDevice", e);
+    return run_attention(ctx, shape, seq, max_len, q, k_cache, v_cache, out, visual_mass, 0, nullptr, nullptr,
+                         nullptr, k_strides, v_strides);
 }
 
 lvspec_status_t lvspec_verify_attention_tree(lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,

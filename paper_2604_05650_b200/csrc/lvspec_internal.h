@@ -38,6 +38,11 @@ struct AttnParams {
     int32_t fp8;
     const float *k_scale;  // [B, Hkv]
     const float *v_scale;  // [B, Hkv]
+    // Cache strides in elements (the head_dim channels of a position are contiguous):
+    // element (b, h, j, c) of k sits at k + b * k_sb + h * k_sh + j * k_sp + c.  The dense
+    // [B, Hkv, Lmax, D] cache has sp = D, sh = Lmax * D, sb = Hkv * Lmax * D; a page pool
+    // [n_pages, Hkv, page_size, D] has sp = D, sh = page_size * D, sb = Hkv * page_size * D.
+    int64_t k_sb, k_sh, k_sp, v_sb, v_sh, v_sp;
 };
 
 // Does draft query `qi` see the cache position with tail index t = pos - (kv_len -

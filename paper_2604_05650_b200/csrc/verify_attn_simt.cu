@@ -80,8 +80,8 @@ attn_simt_kernel(const AttnParams p, const SeqInfo seq)
 #pragma unroll
     for (int i = 0; i < kMaxRowsPerThread; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 
-    const uint16_t *kbase = p.k + ((size_t)b * p.Hkv + kvh) * (size_t)p.Lmax * D;
-    const uint16_t *vbase = p.v + ((size_t)b * p.Hkv + kvh) * (size_t)p.Lmax * D;
+    const uint16_t *kbase = p.k + (size_t)b * p.k_sb + (size_t)kvh * p.k_sh;
+    const uint16_t *vbase = p.v + (size_t)b * p.v_sb + (size_t)kvh * p.v_sh;
     __syncthreads();
 
     for (int t = t_begin; t < t_end; ++t) {
@@ -92,8 +92,8 @@ attn_simt_kernel(const AttnParams p, const SeqInfo seq)
             const int pos = pos0 + j;
             uint4 kk = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
             if (pos < L) {
-                kk = *reinterpret_cast<const uint4 *>(kbase + (size_t)pos * D + c * 8);
-                vv = *reinterpret_cast<const uint4 *>(vbase + (size_t)pos * D + c * 8);
+                kk = *reinterpret_cast<const uint4 *>(kbase + (size_t)pos * p.k_sp + c * 8);
+                vv = *reinterpret_cast<const uint4 *>(vbase + (size_t)pos * p.v_sp + c * 8);
             }
             const uint32_t kw[4] = {kk.x, kk.y, kk.z, kk.w}, vw[4] = {vv.x, vv.y, vv.z, vv.w};
             float *kd = k_s + j * DP + c * 8, *vd = v_s + j * DP + c * 8;

@@ -328,15 +328,16 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
 
     // the cache is read once per call: it should not push the split partials out of L2
     const uint64_t stream_policy = l2_evict_first_policy();
-    // where tile i of this split sits: (position, row of the [.., positions, 128] map)
+    // where tile i of this split sits in the [sequences or pages, heads, positions, 128]
+    // maps: (position, sequence or page)
     volatile int32_t *page_s = reinterpret_cast<volatile int32_t *>(gbase + sm.pages);
     auto tile_at = [&](int i, int &pos0, int &map_row) {
         pos0 = (t_begin + i) * kTilePos;
-        map_row = bh;
+        map_row = b;
         if (kPaged) {
             // a page holds a whole number of tiles; an entry outside the pool reads as zeros
             pos0 -= (pos0 / p.page_size) * p.page_size;
-            map_row = page_s[i] * p.Hkv + kvh;
+            map_row = page_s[i];
         }
     };
     auto load_k = [&](int i) {
@@ -344,9 +345,9 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         int pos0, map_row;
         tile_at(i, pos0, map_row);
         mbar_arrive_expect_tx(k_full(ks), kSlot);
-        tma_load_3d_hint(base + sm.k + ks * kSlot, &tmap_k, k_full(ks), 0, pos0, map_row, stream_policy);
+        tma_load_4d_hint(base + sm.k + ks * kSlot, &tmap_k, k_full(ks), 0, pos0, kvh, map_row, stream_policy);
         if (!kFp8)
-            tma_load_3d_hint(base + sm.k + ks * kSlot + kBoxBytes, &tmap_k, k_full(ks), 64, pos0, map_row,
+            tma_load_4d_hint(base + sm.k + ks * kSlot + kBoxBytes, &tmap_k, k_full(ks), 64, pos0, kvh, map_row,
                              stream_policy);
     };
     auto load_v = [&](int i) {
@@ -354,9 +355,9 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         int pos0, map_row;
         tile_at(i, pos0, map_row);
         mbar_arrive_expect_tx(v_full(vsl), kSlot);
-        tma_load_3d_hint(base + sm.v + vsl * kSlot, &tmap_v, v_full(vsl), 0, pos0, map_row, stream_policy);
+        tma_load_4d_hint(base + sm.v + vsl * kSlot, &tmap_v, v_full(vsl), 0, pos0, kvh, map_row, stream_policy);
         if (!kFp8)
-            tma_load_3d_hint(base + sm.v + vsl * kSlot + kBoxBytes, &tmap_v, v_full(vsl), 64, pos0, map_row,
+            tma_load_4d_hint(base + sm.v + vsl * kSlot + kBoxBytes, &tmap_v, v_full(vsl), 64, pos0, kvh, map_row,
                              stream_policy);
     };
 
@@ -953,32 +954,23 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-// [B*Hkv][Lmax][128] bf16 viewed as a 3-D tensor; boxes of 64 channels x 128 positions
-bool make_kv_map(CUtensorMap *map, const void *ptr, int Lmax, int BH)
+// A cache as a 4-D tensor [sequences or pages][heads][positions][128 channels] with the
+// caller's strides (in elements; the channels are contiguous).  bf16: boxes of 64 channels
+// x 128 positions; E4M3: boxes of 128 channels x 128 positions.
+bool make_kv_map(CUtensorMap *map, const void *ptr, bool fp8, int positions, int heads, int outer,
+                 int64_t s_pos, int64_t s_head, int64_t s_outer)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[3] = {128, (cuuint64_t)Lmax, (cuuint64_t)BH};
-    const cuuint64_t strides[2] = {256, (cuuint64_t)Lmax * 256};
-    const cuuint32_t box[3] = {64, 128, 1};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box,
-              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// [B*Hkv][Lmax][128] E4M3 codes viewed as a 3-D byte tensor; boxes of 128 channels x 128 positions
-bool make_kv_map_fp8(CUtensorMap *map, const void *ptr, int Lmax, int BH)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[3] = {128, (cuuint64_t)Lmax, (cuuint64_t)BH};
-    const cuuint64_t strides[2] = {128, (cuuint64_t)Lmax * 128};
-    const cuuint32_t box[3] = {128, 128, 1};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(ptr), dims, strides, box,
-              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    const cuuint64_t esz = fp8 ? 1 : 2;
+    const cuuint64_t dims[4] = {128, (cuuint64_t)positions, (cuuint64_t)heads, (cuuint64_t)outer};
+    const cuuint64_t strides[3] = {(cuuint64_t)s_pos * esz, (cuuint64_t)s_head * esz, (cuuint64_t)s_outer * esz};
+    const cuuint32_t box[4] = {fp8 ? 128u : 64u, 128, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
+              const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // q [B][gamma][Hq][128] bf16 as a 4-D tensor; one box = 64 channels of the G heads of one
@@ -1041,15 +1033,12 @@ cudaError_t launch_attn_tc(const AttnParams &p, const SeqInfo &seq, cudaStream_t
     if (smem_map(P.cfg).total > kMaxSmem || P.cfg.tmem_cols > 512) return cudaErrorInvalidConfiguration;
     CUtensorMap mk, mv, mq;
     const int map_len = paged ? p.page_size : p.Lmax;
-    const int map_rows = paged ? p.n_pages * p.Hkv : p.B * p.Hkv;
-    if (fp8) {
-        if (!make_kv_map_fp8(&mk, p.k, map_len, map_rows) || !make_kv_map_fp8(&mv, p.v, map_len, map_rows))
-            return cudaErrorInvalidValue;
-        mq = mk;     // not used by the kernel
-    } else if (!make_kv_map(&mk, p.k, map_len, map_rows) || !make_kv_map(&mv, p.v, map_len, map_rows) ||
-               !make_q_map(&mq, p.q, p.B, p.gamma, p.Hq, p.G)) {
+    const int map_outer = paged ? p.n_pages : p.B;
+    if (!make_kv_map(&mk, p.k, fp8, map_len, p.Hkv, map_outer, p.k_sp, p.k_sh, p.k_sb) ||
+        !make_kv_map(&mv, p.v, fp8, map_len, p.Hkv, map_outer, p.v_sp, p.v_sh, p.v_sb))
         return cudaErrorInvalidValue;
-    }
+    if (fp8) mq = mk;     // not used by the kernel
+    else if (!make_q_map(&mq, p.q, p.B, p.gamma, p.Hq, p.G)) return cudaErrorInvalidValue;
     const size_t smem = smem_map(P.cfg).total + 1024;
     const bool tree = p.branch_len != p.gamma;
     if ((tree && paged) || (fp8 && (tree || paged))) return cudaErrorNotSupported;
