@@ -409,6 +409,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 if (i > 0 && i < first_k) load_k(i);
                 load_v(i);
             }
+            for (int i = max(first_v, 1); i < first_k; ++i) load_k(i);    // a K ring deeper than the V ring
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -996,10 +997,13 @@ TcConfig pick_config(int M, int page_slots, bool fp8)
     c.n_pad = (M + 15) & ~15;
     c.page_slots = page_slots;
     c.slot_bytes = fp8 ? kBoxBytes : kSlotBytes;
-    // deepest K/V rings that fit: bytes in flight matter more than a second P buffer,
-    // since the probabilities wait in registers for the buffer anyway (an fp8 tile is
-    // half the bytes: twice the slots for the same bytes in flight)
-    const int tries[6][3] = {{3, 3, 2}, {3, 3, 1}, {2, 3, 2}, {2, 3, 1}, {2, 2, 2}, {2, 2, 1}};
+    // Six ring slots when they fit, also at the price of the second P buffer (with 40 rows
+    // the stream is bound by HBM: bytes in flight count, and the probabilities wait in
+    // registers for the buffer anyway); below that, a second P buffer before a fifth slot
+    // (with 80 rows the chain softmax -> P.V -> next softmax bounds the tile, and two
+    // buffers with 2 + 2 slots beat one with 2 + 3).  An fp8 tile is half the bytes: twice
+    // the slots for the same bytes in flight.
+    const int tries[6][3] = {{3, 3, 2}, {3, 3, 1}, {2, 3, 2}, {2, 2, 2}, {2, 3, 1}, {2, 2, 1}};
     const int tries8[6][3] = {{5, 6, 2}, {5, 5, 2}, {4, 5, 2}, {4, 4, 2}, {4, 4, 1}, {3, 3, 1}};
     for (int t = 0; t < 6; ++t) {
         const int *tr = fp8 ? tries8[t] : tries[t];
