@@ -44,6 +44,10 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch layer by layer, no CUDA graph")
+    ap.add_argument("--fp8-cache", action="store_true",
+                    help="run the step on an fp8 (E4M3) cache with one scale per KV head: the config's caches "
+                         "quantised on the device, lvspec_verify_attention_fp8 in every layer (the roofline then "
+                         "counts one byte per cache element); not the default workload")
     ap.add_argument("--no-other-configs", action="store_true",
                     help="skip the timing of configs 3 and 1 that the default (config 2) run adds to its line")
     ap.add_argument("--no-next-rows", action="store_true",
@@ -302,10 +306,21 @@ class VerifyStep:
     (every layer's attention, then the acceptance pass on the last layer's mass), the
     CUDA graphs they are replayed from, and the device-timed loop."""
 
-    def __init__(self, cfg, ctx, stream, dev, torch, kernel=0, use_graph=True):
+    def __init__(self, cfg, ctx, stream, dev, torch, kernel=0, use_graph=True, fp8=False):
         from paper_2604_05650_b200 import binding
         self.cfg, self.ctx, self.stream, self.dev, self.torch = cfg, ctx, stream, dev, torch
         self.qs, self.ks, self.vs, self.sets = device_workload(cfg, dev, torch)
+        self.fp8 = fp8
+        if fp8:
+            # E4M3 codes and one scale per (sequence, KV head): the largest magnitude -> 448
+            def quantize(t):
+                scale = (t.float().abs().amax(dim=(2, 3)) / 448.0).clamp_min(1e-30)
+                return (t.float() / scale[:, :, None, None]).to(torch.float8_e4m3fn).view(torch.uint8).contiguous(), \
+                    scale.contiguous()
+            self.k8 = [quantize(t) for t in self.ks]
+            self.v8 = [quantize(t) for t in self.vs]
+            self.ks = self.vs = None
+            torch.cuda.empty_cache()
         B, g, Hq, Hkv, D, L = cfg.batch, cfg.gamma, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.kv_len
         self.shape = binding.attn_shape(B, g, Hq, Hkv, D, L, 0, kernel)
         self.kv_len = np.full((B,), L, dtype=np.int32)
@@ -343,8 +358,12 @@ class VerifyStep:
 
     def attention_layers(self):
         for l in range(self.cfg.layers):
-            self.ctx.verify_attention(self.shape, self.qs[l], self.ks[l], self.vs[l], self.kv_len, self.span,
-                                      self.out, self.mass)
+            if self.fp8:
+                self.ctx.verify_attention_fp8(self.shape, self.qs[l], self.k8[l][0], self.v8[l][0], self.k8[l][1],
+                                              self.v8[l][1], self.kv_len, self.span, self.out, self.mass)
+            else:
+                self.ctx.verify_attention(self.shape, self.qs[l], self.ks[l], self.vs[l], self.kv_len, self.span,
+                                          self.out, self.mass)
 
     def accept(self, i):
         c = self.cfg
@@ -402,7 +421,7 @@ class VerifyStep:
 
     def free(self):
         self.graph_attn = self.graph_acc = None
-        self.qs = self.ks = self.vs = self.logits = self.draft = None
+        self.qs = self.ks = self.vs = self.logits = self.draft = self.k8 = self.v8 = None
         self.torch.cuda.empty_cache()
 
 
@@ -413,10 +432,12 @@ def hbm_peak():
     return 6650.0, "fallback", {}
 
 
-def attention_bytes_per_launch(cfg):
-    """Algorithmic bytes of one attention call: K and V once, q and out, the mass."""
+def attention_bytes_per_launch(cfg, fp8=False):
+    """Algorithmic bytes of one attention call: K and V once (one byte per element and the
+    scales with an fp8 cache), q and out, the mass."""
     B, g, Hq, D = cfg.batch, cfg.gamma, cfg.n_q_heads, cfg.head_dim
-    return cfg.kv_bytes_per_layer + 2 * (B * g * Hq * D * 2) + B * g * Hq * 4
+    kv = cfg.kv_bytes_per_layer // 2 + 2 * B * cfg.n_kv_heads * 4 if fp8 else cfg.kv_bytes_per_layer
+    return kv + 2 * (B * g * Hq * D * 2) + B * g * Hq * 4
 
 
 def time_other_config(cfg_id, ctx, stream, dev, torch, args, barrier, local):
@@ -469,7 +490,7 @@ def run_ours(args, cfg):
     ctx = binding.Context(local)
     stream = torch.cuda.Stream(device=dev)
     ctx.set_stream(stream.cuda_stream)
-    vs = VerifyStep(cfg, ctx, stream, dev, torch, args.kernel, not args.no_graph)
+    vs = VerifyStep(cfg, ctx, stream, dev, torch, args.kernel, not args.no_graph, args.fp8_cache)
     B, g, Hq, Hkv, D, L = cfg.batch, cfg.gamma, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.kv_len
 
     ms_total, attn_ms, clock_summary = vs.timed(args.steps, args.warmup, barrier, local)
@@ -483,7 +504,7 @@ def run_ours(args, cfg):
     gpu_mass = vs.mass.cpu().numpy()                   # the last layer's visual mass
 
     # roofline of the dominant kernel: one verification-attention launch
-    bytes_per_launch = attention_bytes_per_launch(cfg)
+    bytes_per_launch = attention_bytes_per_launch(cfg, args.fp8_cache)
     us_per_launch = ms_attn * 1e3 / cfg.layers
     achieved = bytes_per_launch / (us_per_launch * 1e-6) / 1e9
     peak, peak_src, peaks = hbm_peak()
@@ -495,7 +516,7 @@ def run_ours(args, cfg):
         tr = json.load(open(tr_path))
         src = os.path.join(ROOT, tr.get("kernel_source", ""))
         if os.path.exists(src) and hashlib.sha256(open(src, "rb").read()).hexdigest() == tr.get("kernel_source_sha256"):
-            traffic = tr.get(f"config{cfg_id_of(cfg)}")
+            traffic = tr.get(f"config{cfg_id_of(cfg)}" + ("_fp8" if args.fp8_cache else ""))
     # secondary bounds of the same launch: useful tensor flops (two products, 2 flops per
     # multiply-add) against the measured bf16 GEMM rate, and exponentials against the
     # special-function rate (16 per clock and SM at the sampled clock)
@@ -517,7 +538,7 @@ def run_ours(args, cfg):
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": workload_desc(cfg, world),
+            "config": workload_desc(cfg, world), "cache": "e4m3 codes, one scale per KV head" if args.fp8_cache else "bf16",
             "accepted_tokens_per_s": world * accepted / (ms_step * 1e-3),
             "accept_len_mean": accepted, "accept_len_sets": gpu_alen.sum(axis=1).tolist(),
             "accept_sets": f"{N_ACCEPT_SETS} seeded (logits, drafts) sets; step i judges set i mod {N_ACCEPT_SETS}",
@@ -528,19 +549,19 @@ def run_ours(args, cfg):
             "cuda_graph": vs.graph_attn is not None,
             "roofline": roofline, "clocks": clock_summary}
 
-    if not args.no_next_rows and world == 1:
+    if not args.no_next_rows and world == 1 and not args.fp8_cache:
         line["next_rows"] = {"visual_relevance": time_visual_relevance(cfg, ctx, stream, torch, dev, peak, args.top_n),
                              "fp8_attention": time_fp8_attention(cfg, ctx, stream, vs.ks, vs.vs, vs.qs, torch, dev, peak),
                              "paged_attention": time_paged_attention(cfg, ctx, stream, vs.ks, vs.vs, vs.qs, torch, dev, peak),
                              "several_spans": time_span_layer(cfg, ctx, stream, vs.ks, vs.vs, vs.qs, torch, dev)}
 
     # end to end through the host-buffer entry points
-    if not args.no_e2e:
+    if not args.no_e2e and not args.fp8_cache:
         line["e2e"] = run_e2e(args, cfg, ctx, stream, vs, torch, dev, world, barrier, dist)
     sets = vs.sets
     vs.free()
     del vs
-    if world == 1 and not args.no_other_configs and cfg_id_of(cfg) == 2 and args.layers == 0:
+    if world == 1 and not args.no_other_configs and cfg_id_of(cfg) == 2 and args.layers == 0 and not args.fp8_cache:
         line["other_configs"] = {str(i): time_other_config(i, ctx, stream, dev, torch, args, barrier, local)
                                  for i in (3, 1)}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

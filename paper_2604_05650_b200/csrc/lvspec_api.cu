@@ -397,6 +397,16 @@ lvspec_status_t run_accept(lvspec_ctx *ctx, int batch, int gamma, int vocab, int
 
 extern "C" {
 
+#ifdef LVSPEC_TRACE
+// Trace build only (see lvspec_internal.h): where the kernels' time stamps go.
+int lvspec_trace_set_buffer(unsigned long long *device_words)
+{
+    cudaError_t e = trace_set_buffer_attention(device_words);
+    if (e == cudaSuccess) e = trace_set_buffer_merge(device_words);
+    return (int)e;
+}
+#endif
+
 lvspec_status_t lvspec_create(lvspec_ctx_t **out, int device)
 {
     if (!out) {

@@ -5,6 +5,38 @@
 
 #include "lvspec.h"
 
+// Time stamps for performance work, compiled in only with -DLVSPEC_TRACE (a separate
+// build of the library: `python -m paper_2604_05650_b200.trace`; the shipped library has
+// none of it).  The attention and merge kernels then write into a buffer of 64-bit words
+// the caller provides through lvspec_trace_set_buffer (device memory; word 0 counts the
+// records, records of 8 words follow from word 8):
+//   CTA records   {kind (1 attention, 2 merge), q pointer of the call, CTA index,
+//                  %globaltimer at CTA entry, past the prologue / the grid-dependency wait,
+//                  all K.Q^T issued (attention only), end of the CTA's work, unused}
+//   tile records  of the one attention CTA (split 3, KV head 2, sequence 0), from word
+//                 8 + 8 * kTraceCtaRecords on: per role r (0 first softmax warp, 1 K.Q^T
+//                 issuer, 2 P.V issuer), tile i < 32, eight clock64 stamps at
+//                 ((r * 32 + i) * 8): see the LVSPEC_TILE_TS uses in verify_attn_tc.cu
+#ifdef LVSPEC_TRACE
+constexpr int kTraceCtaRecords = 4000;
+// every translation unit with stamps holds its own copy of the buffer address
+static __device__ unsigned long long *g_lvspec_trace = nullptr;
+namespace lvspec {
+cudaError_t trace_set_buffer_attention(unsigned long long *device_words);
+cudaError_t trace_set_buffer_merge(unsigned long long *device_words);
+}
+__device__ __forceinline__ unsigned long long lvspec_trace_now()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+#define LVSPEC_TILE_TS(tr, role, tile, slot) \
+    do { if ((tr) && (tile) < 32) (tr)[(((role) * 32 + (tile)) * 8) + (slot)] = clock64(); } while (0)
+#else
+#define LVSPEC_TILE_TS(tr, role, tile, slot) do { } while (0)
+#endif
+
 namespace lvspec {
 
 // Per-sequence lengths travel as kernel parameters (the C ABI takes them as

@@ -12,6 +12,13 @@
 
 #include "lvspec_internal.h"
 
+#ifdef LVSPEC_TRACE
+cudaError_t lvspec::trace_set_buffer_merge(unsigned long long *device_words)
+{
+    return cudaMemcpyToSymbol(g_lvspec_trace, &device_words, sizeof device_words);
+}
+#endif
+
 namespace lvspec {
 namespace {
 
@@ -218,6 +225,9 @@ __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
 __global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const AttnParams p, const int batch)
 {
     extern __shared__ float4 combine_smem[];
+#ifdef LVSPEC_TRACE
+    const unsigned long long trace_t0 = lvspec_trace_now();
+#endif
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // every address is worked out before the wait for the attention grid: the CTA is
     // resident by then, and the cold parameter loads and index arithmetic cost it nothing
@@ -239,6 +249,20 @@ __global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const 
     float *mass_row = p.mass + row;
     float *lse_row = p.lse2 ? p.lse2 + row : nullptr;
     asm volatile("griddepcontrol.wait;" ::: "memory");
+#ifdef LVSPEC_TRACE
+    unsigned long long *rec = nullptr;
+    if (g_lvspec_trace && threadIdx.x == 0) {
+        const unsigned long long idx = atomicAdd(g_lvspec_trace, 1ull);
+        if (idx < (unsigned long long)kTraceCtaRecords) {
+            rec = g_lvspec_trace + 8 + idx * 8;
+            rec[0] = 2;
+            rec[1] = (unsigned long long)p.q;
+            rec[2] = blockIdx.x + 1000 * blockIdx.y + 1000000 * blockIdx.z;
+            rec[3] = trace_t0;
+            rec[4] = lvspec_trace_now();
+        }
+    }
+#endif
 
     float m_run = -INFINITY, l = 0.f, lv = 0.f;
     float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -305,6 +329,9 @@ __global__ void __launch_bounds__(32 * kCombineWarps) attn_combine_kernel(const 
         *mass_row = lv * inv;
         if (lse_row) *lse_row = m_run + log2f(l);
     }
+#ifdef LVSPEC_TRACE
+    if (rec) rec[6] = lvspec_trace_now();
+#endif
 }
 
 }  // namespace

@@ -50,6 +50,13 @@
 #include "lvspec_internal.h"
 #include "sm100_ptx.cuh"
 
+#ifdef LVSPEC_TRACE
+cudaError_t lvspec::trace_set_buffer_attention(unsigned long long *device_words)
+{
+    return cudaMemcpyToSymbol(g_lvspec_trace, &device_words, sizeof device_words);
+}
+#endif
+
 namespace lvspec {
 namespace {
 
@@ -267,6 +274,24 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     const AttnParams &p = P.a;
     const TcConfig cfg = P.cfg;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef LVSPEC_TRACE
+    unsigned long long *rec = nullptr;      // this CTA's record (one thread writes it)
+    long long *tile_tr = nullptr;           // per-tile stamps of the one traced CTA (lane 0 of its warps)
+    if (g_lvspec_trace && tid == 32) {
+        const unsigned long long idx = atomicAdd(g_lvspec_trace, 1ull);
+        if (idx < (unsigned long long)kTraceCtaRecords) {
+            rec = g_lvspec_trace + 8 + idx * 8;
+            rec[0] = 1;
+            rec[1] = (unsigned long long)P.a.q;
+            rec[2] = blockIdx.x + 1000 * blockIdx.y + 1000000 * blockIdx.z;
+            rec[3] = lvspec_trace_now();
+        }
+    }
+    if (g_lvspec_trace && blockIdx.x == 3 && blockIdx.y == 2 && blockIdx.z == 0 && lane == 0)
+        tile_tr = reinterpret_cast<long long *>(g_lvspec_trace + 8 + 8 * kTraceCtaRecords);
+#else
+    constexpr long long *tile_tr = nullptr;
+#endif
     // the TMA unit fetches the descriptors while everything else is set up; a warp that
     // has nothing to do in the prologue asks for them, not the producer (whose first
     // load is what the whole CTA waits for)
@@ -475,6 +500,9 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+#ifdef LVSPEC_TRACE
+    if (rec) rec[4] = lvspec_trace_now();
+#endif
     const uint32_t tmem_base = *tmem_slot;
     // accumulator columns: S^T twice, then O^T and the sums (fp8 cache: two columns per row)
     constexpr int kAccCols = kFp8 ? 2 : 1;
@@ -605,8 +633,11 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                                        kSwizzle128B);
             auto issue_qk = [&](int i) -> bool {
                 const int ks = i % cfg.ks, sb = i & 1;
+                LVSPEC_TILE_TS(tile_tr, 1, i, 0);     // starts waiting for the K tile
                 if (!mbar_wait(k_full(ks), (i / cfg.ks) & 1, abort_flag)) return false;
+                LVSPEC_TILE_TS(tile_tr, 1, i, 1);     // K tile there
                 if (i >= 2 && !mbar_wait(s_free(sb), ((i >> 1) - 1) & 1, abort_flag)) return false;
+                LVSPEC_TILE_TS(tile_tr, 1, i, 2);     // S^T buffer free
                 tc_fence_after();
                 const uint64_t kd = kd0 + (uint64_t)(ks * (kSlot >> 4));
                 const uint32_t d = tm_s0 + sb * NP;
@@ -620,6 +651,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 }
                 mma_commit(s_full(sb));
                 mma_commit(k_empty(ks));
+                LVSPEC_TILE_TS(tile_tr, 1, i, 3);     // K.Q^T issued
                 return true;
             };
             bool ok = mbar_wait(q_full, 0, abort_flag);
@@ -641,8 +673,11 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             const uint64_t a2d0 = make_smem_desc(base + sm.a2, 1024, 128, kSwizzleNone);
             for (int i = 0; i < T; ++i) {
                 const int pb = i % cfg.pb, vsl = i % cfg.vs;
+                LVSPEC_TILE_TS(tile_tr, 2, i, 0);     // starts waiting for P^T
                 if (!mbar_wait(p_full(pb), (i / cfg.pb) & 1, abort_flag)) break;
+                LVSPEC_TILE_TS(tile_tr, 2, i, 1);     // P^T there
                 if (!mbar_wait(v_full(vsl), (i / cfg.vs) & 1, abort_flag)) break;
+                LVSPEC_TILE_TS(tile_tr, 2, i, 2);     // V tile there
                 tc_fence_after();
                 // V^T: channels contiguous (M-major), 64-channel halves kBoxBytes apart,
                 // groups of 8 positions 1024 bytes apart.  P^T: rows contiguous in
@@ -683,6 +718,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 }
                 mma_commit(v_empty(vsl));
                 mma_commit(p_free(pb));
+                LVSPEC_TILE_TS(tile_tr, 2, i, 3);     // sums and P.V issued
             }
             // this thread's MMAs have finished: tell the TMEM owner
             mma_commit(done_bar);
@@ -708,7 +744,9 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             const int pos0 = (t_begin + i) * kTilePos;
             const int pos = pos0 + row;
             const int sb = i & 1;
+            if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 0);     // starts waiting for S^T
             mbar_wait(s_full(sb), (i >> 1) & 1, abort_flag);
+            if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 1);     // S^T there
             tc_fence_after();
             const uint32_t s_addr = tm_s0 + sb * NP + lane_addr;
             if (!kFp8 && i == 0) {
@@ -740,6 +778,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                     const float gmax =
                         !tail ? softmax_pass<0, kFp8>(s_addr, c_lo, c_hi, m_s, scale, vis_s, G, gmin, pk)
                               : softmax_pass<kTree ? 2 : 1, kFp8>(s_addr, c_lo, c_hi, m_s, scale, vis_s, G, gmin, pk);
+                    if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 2);     // exponentials done
                     if (!group_any(bar_id, gmax > kLimit)) break;
                 }
 
@@ -813,8 +852,10 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                     }
                 }
             }
+            if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 3);     // the group agrees: no rescale
             // P^T goes to shared memory once the P.V product that read this buffer is done
             if (pb_round > 0) mbar_wait(p_free(pb), (pb_round - 1) & 1, abort_flag);
+            if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 4);     // P buffer free
 #pragma unroll
             for (int j = 0; j < kMaxChunks; ++j)
                 if (c_lo + j < c_hi) *reinterpret_cast<uint4 *>(prow + (c_lo + j) * 2048) = pk[j];
@@ -827,6 +868,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 mbar_arrive(s_free(sb));
                 mbar_arrive(p_full(pb));
             }
+            if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 5);     // P^T stored and handed over
             if (++pb == cfg.pb) { pb = 0; ++pb_round; }
             if (++vsl == cfg.vs) { vsl = 0; ++vs_round; }
         }
@@ -923,7 +965,13 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     if (warp == 1) {
         if (lane == 0) {
             bool all_done = false;
+#ifdef LVSPEC_TRACE
+            if (rec) rec[5] = lvspec_trace_now();
+#endif
             for (int tries = 0; tries < 4 && !all_done; ++tries) all_done = wait_unconditional(done_bar, 0);
+#ifdef LVSPEC_TRACE
+            if (rec) rec[6] = lvspec_trace_now();
+#endif
             if (*abort_flag || !all_done) atomicOr(p.status, LVSPEC_DEV_WAIT_EXPIRED);
             // this CTA is done but for freeing TMEM: a dependent launch may be scheduled
             // once every CTA has come this far (earlier, its CTAs would pile up on the
