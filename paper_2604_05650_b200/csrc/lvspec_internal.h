@@ -15,7 +15,7 @@
 //                  all K.Q^T issued (attention only), end of the CTA's work, unused}
 //   tile records  of the one attention CTA (split 3, KV head 2, sequence 0), from word
 //                 8 + 8 * kTraceCtaRecords on: per role r (0 first softmax warp, 1 K.Q^T
-//                 issuer, 2 P.V issuer), tile i < 32, eight clock64 stamps at
+//                 issuer, 2 P.V issuer, 3 inside the first softmax warp's pass), tile i < 32, eight clock64 stamps at
 //                 ((r * 32 + i) * 8): see the LVSPEC_TILE_TS uses in verify_attn_tc.cu
 #ifdef LVSPEC_TRACE
 constexpr int kTraceCtaRecords = 4000;

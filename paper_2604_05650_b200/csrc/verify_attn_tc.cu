@@ -22,9 +22,17 @@
 // K.Q^T MMAs and TMEM owner, warp 14 = issuer of the P.V and sum MMAs (one
 // thread each; two issuers because a single thread's issue rate, not the tensor
 // pipe, bounded the loop), warps 2-13 = three softmax groups of four warps.
-// All groups work on every tile, each on its own share of the N columns (TMEM
-// lane quarter = warp % 4), so the shares never interact: each has its own m,
-// its own guard and its own rescale.  K and V tiles sit in separate shared-memory rings,
+// The groups take the tiles in turn (tile i belongs to group i % 3; a thread is
+// one cache position, TMEM lane quarter = warp % 4, and works through all N
+// columns of its tile), so the latencies of one tile (TMEM load, barrier,
+// hand-over) hide behind the exponentials of the two tiles the other groups are
+// on; S^T has a TMEM buffer per tile in flight.  The reference exponents m[] are
+// shared.  Tiles are handed to the P.V issuer strictly in order, through a
+// counter of committed tiles: a group may move m (and rescale the accumulators)
+// only while its tile is the oldest uncommitted one, and announces the move in an
+// epoch counter; a group whose turn comes compares the epoch with the one it read
+// m under and computes its tile once more if m has moved meanwhile.
+// K and V tiles sit in separate shared-memory rings,
 // each slot two 128-position x 64-channel boxes with the 128-byte swizzle; Q
 // arrives by TMA in the same layout.  Every mbarrier wait is bounded; a wait
 // that gives up raises LVSPEC_DEV_WAIT_EXPIRED.
@@ -46,6 +54,10 @@
 // epilogue.
 #include <cuda.h>
 #include <cuda_bf16.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <type_traits>
 
 #include "lvspec_internal.h"
 #include "sm100_ptx.cuh"
@@ -69,13 +81,13 @@ constexpr int kSoftmaxWarps = 4 * kSoftmaxGroups;
 constexpr int kSoftmaxThreads = 32 * kSoftmaxWarps;
 constexpr int kPvWarp = kSoftmaxWarp0 + kSoftmaxWarps;   // issues the P.V and sum MMAs
 constexpr int kThreads = 32 * (kPvWarp + 1);
-constexpr int kMaxChunks = (LVSPEC_MAX_ROWS / 8 + kSoftmaxGroups - 1) / kSoftmaxGroups;   // per group
+constexpr int kMaxChunks = (LVSPEC_MAX_ROWS / 8 + kSoftmaxGroups - 1) / kSoftmaxGroups;   // per group that shares the columns
 constexpr uint32_t kBoxBytes = 16384;       // 128 positions x 64 channels bf16, or x 128 channels E4M3
 constexpr uint32_t kSlotBytes = 2 * kBoxBytes;   // a bf16 tile; an fp8 tile is one box
 constexpr uint32_t kA2Bytes = 2048;         // one 64 x 16 (bf16) or 64 x 32 (E4M3) constant tile
 constexpr float kGuard = 60.f;              // log2 units above m before a rescale
 constexpr float kGuard8 = 8.f;              // fp8 cache: probabilities stay below 2^8 (E4M3 ends at 448)
-constexpr float kHead8 = 5.f;               // fp8 cache: the score a row's reference is taken from has probability 2^5
+constexpr float kHead8 = 3.f;               // fp8 cache: the largest score of a row in the split's first tile has probability 2^3
 constexpr float kMFloor = -1.0e30f;
 constexpr int kQBarrier = 1 + kSoftmaxGroups;   // named barrier over all softmax threads
 constexpr int kMaxRowsFp8 = 80;             // fp8 cache: 6 accumulator columns per padded row in 512
@@ -83,6 +95,7 @@ constexpr int kMaxRowsFp8 = 80;             // fp8 cache: 6 accumulator columns 
 struct TcConfig {
     int n_pad;   // MMA N: rows padded to a multiple of 16
     int ks, vs, pb;   // K slots, V slots, P buffers
+    int sb;           // S^T buffers in TMEM (2 or 3)
     int tmem_cols;
     int page_slots;   // paged cache: pool pages of this split's tiles, one entry per tile
     int slot_bytes;   // one K or V tile: 32 KB bf16, 16 KB fp8
@@ -105,8 +118,8 @@ __host__ __device__ inline SmemMap smem_map(const TcConfig &c)
     s.dl = o;   o += c.n_pad * 4;
     s.tmx = o;  o += 4 * c.n_pad * 4;
     s.vis = o;  o += c.n_pad * 8;
-    s.bars = o; o += 8 * (2 * c.ks + 2 * c.vs + 4 + 2 * c.pb + 3);
-    s.misc = o; o += 16 + 4 * kSoftmaxWarps;     // TMEM address, abort flag, per-warp maxima of |q|
+    s.bars = o; o += 8 * (2 * c.ks + 2 * c.vs + 4 * kSoftmaxGroups + 4);
+    s.misc = o; o += 16 + 4 * kSoftmaxWarps;     // TMEM address, abort flag, epoch of m, committed tiles, per-warp maxima of |q|
     s.pages = o; o += 4 * c.page_slots;
     s.total = o;
     return s;
@@ -115,6 +128,21 @@ __host__ __device__ inline SmemMap smem_map(const TcConfig &c)
 struct TcParams {
     AttnParams a;
     TcConfig cfg;
+};
+
+// Position in a ring of n slots and the parity of the round: the per-tile loops count
+// instead of dividing.
+struct Ring {
+    int idx, n;
+    uint32_t parity;
+    __device__ __forceinline__ Ring(int n_) : idx(0), n(n_), parity(0) {}
+    __device__ __forceinline__ void next()
+    {
+        if (++idx == n) {
+            idx = 0;
+            parity ^= 1u;
+        }
+    }
 };
 
 __device__ __forceinline__ bool wait_unconditional(uint32_t bar, uint32_t parity)
@@ -231,12 +259,47 @@ __device__ __forceinline__ float exp_chunk(const uint32_t (&r)[8], const float *
     return mx;
 }
 
-// One pass over this thread's position: exp2 of its chunks [c_lo, c_hi) of S^T (up to
+// One pass over this thread's position: exp2 of all n8 column chunks of S^T (four TMEM
+// loads in flight per wait), the packed probabilities stored to this position's place in
+// the P^T buffer; returns the largest scaled score.  kMask != 0: the tile reaches into the
+// draft slots, so columns are masked by what their query may see; the common tile carries
+// none of that.  The loop stays rolled: three groups run it at different places, and
+// the instruction cache holds the short form better.
+template <int kMask, bool kFp8>
+__device__ __forceinline__ float softmax_pass(uint32_t s_addr, int n8, const float *m_s, float scale,
+                                              const int2 *vis_s, int G, int t, uint8_t *prow, long long *tr,
+                                              int tile)
+{
+    float gmax = -INFINITY;
+#pragma unroll 1
+    for (int cb = 0; cb < n8; cb += 4) {
+        uint32_t r[4][8];
+        LVSPEC_TILE_TS(tr, 3, tile, (cb >> 2) * 3);         // asks for four chunks of S^T
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (cb + u < n8) tmem_ld_x8(s_addr + (cb + u) * 8, r[u]);
+        tmem_wait_ld();
+        LVSPEC_TILE_TS(tr, 3, tile, (cb >> 2) * 3 + 1);     // has them
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (cb + u < n8) {
+                uint4 pk;
+                gmax = fmaxf(gmax, exp_chunk<kMask, kFp8>(r[u], m_s + (cb + u) * 8, scale, vis_s + (cb + u) * 8,
+                                                          (cb + u) * 8, G, t, pk));
+                *reinterpret_cast<uint4 *>(prow + (cb + u) * 2048) = pk;
+            }
+        LVSPEC_TILE_TS(tr, 3, tile, (cb >> 2) * 3 + 2);     // their probabilities stored
+    }
+    return gmax;
+}
+
+// The same for a group that works on a share of the columns, chunks [c_lo, c_hi), of every
+// tile: exp2 of its chunks of S^T (up to
 // four TMEM loads in flight per wait), packed probabilities into pk, returns the
 // largest scaled score.  kMask != 0: the tile reaches into the draft slots, so
 // columns are masked by what their query may see; the common tile carries none of that.
 template <int kMask, bool kFp8>
-__device__ __forceinline__ float softmax_pass(uint32_t s_addr, int c_lo, int c_hi, const float *m_s,
+__device__ __forceinline__ float softmax_pass_share(uint32_t s_addr, int c_lo, int c_hi, const float *m_s,
                                               float scale, const int2 *vis_s, int G, int t,
                                               uint4 (&pk)[kMaxChunks])
 {
@@ -259,12 +322,15 @@ __device__ __forceinline__ float softmax_pass(uint32_t s_addr, int c_lo, int c_h
     }
     return gmax;
 }
-
 // kTree: the draft slots hold several branches (the visibility table is only built
 // and read then; the plain chain keeps its arithmetic mask).  kPaged: K and V are page
 // pools and a tile's position in them comes from the sequence's block table.
 // kFp8: E4M3 cache (tmap_q is not used: q is split into its two E4M3 tiles by the CTA).
-template <bool kTree, bool kPaged, bool kFp8>
+// kTurns: the softmax groups take the tiles in turn; otherwise all groups work on every
+// tile, each on a share of its columns (shorter per tile, and so at the two ends of a
+// CTA's stream, but the per-tile overheads are paid by all twelve warps: the form for few
+// query rows, where the stream is bound by HBM either way).
+template <bool kTree, bool kPaged, bool kFp8, bool kTurns>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUtensorMap tmap_k,
                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_q)
@@ -288,7 +354,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         }
     }
     if (g_lvspec_trace && blockIdx.x == 3 && blockIdx.y == 2 && blockIdx.z == 0 && lane == 0)
-        tile_tr = reinterpret_cast<long long *>(g_lvspec_trace + 8 + 8 * kTraceCtaRecords);
+        tile_tr = reinterpret_cast<long long *>(g_lvspec_trace + 8 + 8 * kTraceCtaRecords);   // 4 roles x 32 tiles x 8 stamps
 #else
     constexpr long long *tile_tr = nullptr;
 #endif
@@ -334,6 +400,9 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     int2 *vis_s = reinterpret_cast<int2 *>(gbase + sm.vis);
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gbase + sm.misc);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(gbase + sm.misc + 4);
+    // how often the reference exponents m[] have been set or moved; tiles handed to the P.V issuer
+    volatile uint32_t *epoch_s = reinterpret_cast<volatile uint32_t *>(gbase + sm.misc + 8);
+    volatile uint32_t *committed_s = reinterpret_cast<volatile uint32_t *>(gbase + sm.misc + 12);
 
     // barrier addresses
     const uint32_t bar0 = base + sm.bars;
@@ -342,13 +411,19 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     auto v_full = [&](int s) { return bar0 + 8 * (2 * cfg.ks + s); };
     auto v_empty = [&](int s) { return bar0 + 8 * (2 * cfg.ks + cfg.vs + s); };
     const uint32_t bar1 = bar0 + 8 * (2 * cfg.ks + 2 * cfg.vs);
-    auto s_full = [&](int s) { return bar1 + 8 * s; };
-    auto s_free = [&](int s) { return bar1 + 8 * (2 + s); };
-    auto p_full = [&](int s) { return bar1 + 8 * (4 + s); };
-    auto p_free = [&](int s) { return bar1 + 8 * (4 + cfg.pb + s); };
-    const uint32_t drain_bar = bar1 + 8 * (4 + 2 * cfg.pb);
+    // The hand-over barriers of tile i are those of index i % 3, whatever the number of
+    // S^T and P^T buffers: a parity wait tells a phase from its neighbours only, so whoever
+    // waits for a phase must know the phase before it to be over.  Each of these
+    // barriers belongs to the tiles of one softmax group, which sees its phases in order.
+    auto s_full = [&](int i) { return bar1 + 8 * (i % kSoftmaxGroups); };
+    auto s_free = [&](int i) { return bar1 + 8 * (kSoftmaxGroups + i % kSoftmaxGroups); };
+    auto p_full = [&](int i) { return bar1 + 8 * (2 * kSoftmaxGroups + i % kSoftmaxGroups); };
+    auto p_free = [&](int i) { return bar1 + 8 * (3 * kSoftmaxGroups + i % kSoftmaxGroups); };
+    auto hand_parity = [](int i) { return (uint32_t)(i / kSoftmaxGroups) & 1u; };
+    const uint32_t drain_bar = bar1 + 8 * (4 * kSoftmaxGroups);
     const uint32_t done_bar = drain_bar + 8;
     const uint32_t q_full = drain_bar + 16;
+    const uint32_t pv_done = drain_bar + 24;
     const int bh = b * p.Hkv + kvh;
 
     // the cache is read once per call: it should not push the split partials out of L2
@@ -394,18 +469,23 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         {
             // one barrier per lane, all at once (an mbarrier.init costs about a hundred
             // cycles): barriers sit in the order k_full, k_empty, v_full, v_empty,
-            // s_full[2], s_free[2], p_full, p_free, drain, done, q_full
+            // s_full[3], s_free[3], p_full[3], p_free[3], drain, done, q_full, pv_done
             const int n_kv = 2 * cfg.ks + 2 * cfg.vs;
-            const int n_bars = n_kv + 4 + 2 * cfg.pb + 3;
+            constexpr int n_sp = 4 * kSoftmaxGroups;
+            const int n_bars = n_kv + n_sp + 4;
             for (int i = lane; i < n_bars; i += 32) {
                 const int j = i - n_kv;          // index among the barriers after the rings
                 uint32_t count = 1;
-                if (j >= 2 && j < 4 + cfg.pb) count = kSoftmaxWarps;           // s_free, p_full
-                else if (j == 4 + 2 * cfg.pb + 1) count = kSoftmaxWarps + 1;   // done
-                else if (kFp8 && j == 4 + 2 * cfg.pb + 2) count = kSoftmaxWarps;   // q_full: the warps that split q
+                if (j >= kSoftmaxGroups && j < 3 * kSoftmaxGroups) count = kTurns ? 4 : kSoftmaxWarps;   // s_free, p_full: the warps that work on a tile
+                else if (j == n_sp + 1) count = kSoftmaxWarps + 1;              // done
+                else if (kFp8 && j == n_sp + 2) count = kSoftmaxWarps;          // q_full: the warps that split q
                 mbar_init(bar0 + 8 * i, count);
             }
-            if (lane == 0) *abort_flag = 0;
+            if (lane == 0) {
+                *abort_flag = 0;
+                *epoch_s = 0;
+                *committed_s = 0;
+            }
             mbar_fence_init();
             fence_proxy_async_smem();
         }
@@ -504,9 +584,9 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     if (rec) rec[4] = lvspec_trace_now();
 #endif
     const uint32_t tmem_base = *tmem_slot;
-    // accumulator columns: S^T twice, then O^T and the sums (fp8 cache: two columns per row)
+    // accumulator columns: the S^T buffers, then O^T and the sums (fp8 cache: two columns per row)
     constexpr int kAccCols = kFp8 ? 2 : 1;
-    const uint32_t tm_s0 = tmem_base, tm_o = tmem_base + 2 * NP, tm_l = tm_o + kAccCols * NP;
+    const uint32_t tm_s0 = tmem_base, tm_o = tmem_base + cfg.sb * NP, tm_l = tm_o + kAccCols * NP;
     float scale_cta = p.scale_log2;     // softmax scale of this CTA (fp8 cache: with the K scale and q's shift)
     float v_scale = 1.f;
     if (kFp8 && warp >= kSoftmaxWarp0 && warp < kPvWarp) {
@@ -621,7 +701,10 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         }
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
+        // The whole warp runs the loop and one elected lane issues: the descriptors are
+        // then the same in every lane and the compiler can keep them where the MMA
+        // instruction takes its operands from, instead of moving them there per instruction.
+        {
             const uint32_t idesc_qk = kFp8 ? make_idesc_e4m3(128, NP, 0, 0) : make_idesc_bf16(128, NP, 0, 0);
             // descriptors: everything but the start address is fixed, and the start
             // address field (address / 16) moves by compile-time steps
@@ -631,38 +714,54 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             for (int j = 0; j < 8; ++j)
                 qd[j] = make_smem_desc(base + sm.q + (j >> 2) * (NP * 128) + (j & 3) * 32, 16, 1024,
                                        kSwizzle128B);
+            Ring k_ring(cfg.ks), s_ring(cfg.sb), hand(kSoftmaxGroups), freed(kSoftmaxGroups);
             auto issue_qk = [&](int i) -> bool {
-                const int ks = i % cfg.ks, sb = i & 1;
+                const int ks = k_ring.idx, sb = s_ring.idx;
                 LVSPEC_TILE_TS(tile_tr, 1, i, 0);     // starts waiting for the K tile
-                if (!mbar_wait(k_full(ks), (i / cfg.ks) & 1, abort_flag)) return false;
+                bool there = mbar_wait(k_full(ks), k_ring.parity, abort_flag);
                 LVSPEC_TILE_TS(tile_tr, 1, i, 1);     // K tile there
-                if (i >= 2 && !mbar_wait(s_free(sb), ((i >> 1) - 1) & 1, abort_flag)) return false;
+                // the tile that used this S^T buffer last (tile i - sb) has been read
+                if (i >= cfg.sb) {
+                    there = mbar_wait(bar1 + 8 * (kSoftmaxGroups + freed.idx), freed.parity, abort_flag) && there;
+                    freed.next();
+                }
+                if (!__all_sync(0xffffffffu, there)) return false;
                 LVSPEC_TILE_TS(tile_tr, 1, i, 2);     // S^T buffer free
                 tc_fence_after();
                 const uint64_t kd = kd0 + (uint64_t)(ks * (kSlot >> 4));
                 const uint32_t d = tm_s0 + sb * NP;
                 // bf16: 8 steps of 16 channels over the two 64-channel boxes; fp8: 4 steps of
                 // 32 channels against q's leading bits, then the same 4 against the rest
+                if (elect_one()) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    if (kFp8) mma_f8_ss(d, kd + (uint64_t)((j & 3) * 2), qd[j], idesc_qk, j > 0);
-                    else mma_f16_ss(d, kd + (uint64_t)((j >> 2) * (kBoxBytes >> 4) + (j & 3) * 2), qd[j],
-                                    idesc_qk, j > 0);
+                    for (int j = 0; j < 8; ++j) {
+                        if (kFp8) mma_f8_ss(d, kd + (uint64_t)((j & 3) * 2), qd[j], idesc_qk, j > 0);
+                        else mma_f16_ss(d, kd + (uint64_t)((j >> 2) * (kBoxBytes >> 4) + (j & 3) * 2), qd[j],
+                                        idesc_qk, j > 0);
+                    }
+                    mma_commit(bar1 + 8 * hand.idx);      // s_full of tile i
+                    mma_commit(k_empty(ks));
                 }
-                mma_commit(s_full(sb));
-                mma_commit(k_empty(ks));
+                __syncwarp();
                 LVSPEC_TILE_TS(tile_tr, 1, i, 3);     // K.Q^T issued
+                k_ring.next();
+                s_ring.next();
+                hand.next();
                 return true;
             };
-            bool ok = mbar_wait(q_full, 0, abort_flag);
+            bool ok = __all_sync(0xffffffffu, mbar_wait(q_full, 0, abort_flag));
             for (int i = 0; ok && i < T; ++i) ok = issue_qk(i);
-            // every MMA issued by this thread has finished before TMEM is released
-            mma_commit(drain_bar);
-            wait_unconditional(drain_bar, 0);
+            // every MMA issued by the elected lane has finished before TMEM is released
+            if (elect_one()) {
+                mma_commit(drain_bar);
+                wait_unconditional(drain_bar, 0);
+            }
+            __syncwarp();
         }
     } else if (warp == kPvWarp) {
         // ------------------------------------------------- P.V and sum MMA issuer
-        if (lane == 0) {
+        // (whole warp in the loop, one elected lane issues: see the K.Q^T issuer)
+        {
             const uint32_t idesc_pv = kFp8 ? make_idesc_e4m3(128, 2 * NP, 1, 1) : make_idesc_bf16(128, NP, 1, 1);
             const uint32_t idesc_sum = kFp8 ? make_idesc_e4m3(64, 2 * NP, 0, 1) : make_idesc_bf16(64, NP, 0, 1);
             // one MMA covers 16 positions of a bf16 tile, 32 of an fp8 tile
@@ -671,12 +770,14 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             const uint64_t vd0 = make_smem_desc(base + sm.v, kBoxBytes, 1024, kSwizzle128B);
             const uint64_t pd0 = make_smem_desc(base + sm.p, 128, 2048, kSwizzleNone);
             const uint64_t a2d0 = make_smem_desc(base + sm.a2, 1024, 128, kSwizzleNone);
-            for (int i = 0; i < T; ++i) {
-                const int pb = i % cfg.pb, vsl = i % cfg.vs;
+            Ring v_ring(cfg.vs), p_ring(cfg.pb), hand(kSoftmaxGroups);
+            for (int i = 0; i < T; ++i, v_ring.next(), p_ring.next(), hand.next()) {
+                const int pb = p_ring.idx, vsl = v_ring.idx;
                 LVSPEC_TILE_TS(tile_tr, 2, i, 0);     // starts waiting for P^T
-                if (!mbar_wait(p_full(pb), (i / cfg.pb) & 1, abort_flag)) break;
+                bool there = mbar_wait(bar1 + 8 * (2 * kSoftmaxGroups + hand.idx), hand.parity, abort_flag);   // p_full of tile i
                 LVSPEC_TILE_TS(tile_tr, 2, i, 1);     // P^T there
-                if (!mbar_wait(v_full(vsl), (i / cfg.vs) & 1, abort_flag)) break;
+                there = mbar_wait(v_full(vsl), v_ring.parity, abort_flag) && there;
+                if (!__all_sync(0xffffffffu, there)) break;
                 LVSPEC_TILE_TS(tile_tr, 2, i, 2);     // V tile there
                 tc_fence_after();
                 // V^T: channels contiguous (M-major), 64-channel halves kBoxBytes apart,
@@ -692,7 +793,9 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 if (pos0 >= vs && pos0 + kTilePos <= ve) uniform = 0;
                 else if (pos0 + kTilePos <= vs || pos0 >= ve) uniform = 1;
                 const uint32_t first_acc = i > 0 ? 1u : 0u;
-                if (uniform >= 0) {
+                if (!elect_one()) {
+                    // the other lanes wait at the end of the turn
+                } else if (uniform >= 0) {
                     const uint64_t d2 = a2d0 + (uint64_t)(uniform * (kA2Bytes >> 4));
 #pragma unroll
                     for (int j = 0; j < kSteps; ++j)
@@ -716,169 +819,383 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                                      pd + (uint64_t)(j * kPStep), idesc_sum, acc);
                     }
                 }
-                mma_commit(v_empty(vsl));
-                mma_commit(p_free(pb));
+                if (elect_one()) {
+                    mma_commit(v_empty(vsl));
+                    mma_commit(bar1 + 8 * (3 * kSoftmaxGroups + hand.idx));     // p_free of tile i
+                }
+                __syncwarp();
                 LVSPEC_TILE_TS(tile_tr, 2, i, 3);     // sums and P.V issued
             }
-            // this thread's MMAs have finished: tell the TMEM owner
-            mma_commit(done_bar);
+            // the elected lane's MMAs have finished: tell the softmax warps and the TMEM owner
+            if (elect_one()) {
+                mma_commit(pv_done);
+                mma_commit(done_bar);
+            }
+            __syncwarp();
         }
     } else {
         // ------------------------------------------------------------ softmax warps
-        const int grp = (warp - kSoftmaxWarp0) >> 2;    // column half this warp works on
+        const int grp = (warp - kSoftmaxWarp0) >> 2;    // tiles grp, grp + 3, ... are this group's
         const int bar_id = 1 + grp;
         const int wq = warp & 3;                        // TMEM lane quarter of this warp
         const int row = wq * 32 + lane;                 // TMEM lane = position inside the tile
         const int gtid = ((warp - kSoftmaxWarp0) & 3) * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
-        // chunks of 8 columns [c_lo, c_hi) of this group: equal shares, at most kMaxChunks
-        const int c_base = n8 / kSoftmaxGroups, c_rem = n8 - c_base * kSoftmaxGroups;
-        const int c_lo = grp * c_base + min(grp, c_rem), c_hi = c_lo + c_base + (grp < c_rem ? 1 : 0);
         const float scale = scale_cta;
         constexpr float kLimit = kFp8 ? kGuard8 : kGuard;    // a score this far above m moves m
         constexpr float kLift = kFp8 ? kHead8 : 0.f;         // where the reference position sits above m
-        // ring positions advance by counting, not by dividing
-        int pb = 0, vsl = 0;                 // P buffer and V slot of tile i
-        uint32_t pb_round = 0, vs_round = 0; // how often each ring has wrapped
-        for (int i = 0; i < T; ++i) {
-            const int pos0 = (t_begin + i) * kTilePos;
-            const int pos = pos0 + row;
-            const int sb = i & 1;
-            if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 0);     // starts waiting for S^T
-            mbar_wait(s_full(sb), (i >> 1) & 1, abort_flag);
-            if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 1);     // S^T there
-            tc_fence_after();
-            const uint32_t s_addr = tm_s0 + sb * NP + lane_addr;
-            if (!kFp8 && i == 0) {
-                // reference exponent of each row: its score at the split's first position
-                if (wq == 0) {
-                    for (int c8 = c_lo; c8 < c_hi; ++c8) {
-                        uint32_t r[8];
-                        tmem_ld_x8(s_addr + c8 * 8, r);
-                        tmem_wait_ld();
-                        if (lane == 0) {
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) m_s[c8 * 8 + k] = __uint_as_float(r[k]) * scale - kLift;
+        // this group's share of the columns (all tiles without turns; the epilogue always):
+        // chunks of 8 columns [c_lo, c_hi), equal shares, at most kMaxChunks
+        const int c_base = n8 / kSoftmaxGroups, c_rem = n8 - c_base * kSoftmaxGroups;
+        const int c_lo = grp * c_base + min(grp, c_rem), c_hi = c_lo + c_base + (grp < c_rem ? 1 : 0);
+        if constexpr (kTurns) {
+            // bounded wait for a shared-memory counter to reach a value (the groups' turns)
+            auto wait_counter = [&](volatile uint32_t *ctr, uint32_t at_least) {
+                if (*ctr >= at_least) return;
+                uint64_t t0 = 0;
+                for (uint32_t spin = 1;; ++spin) {
+                    if (*ctr >= at_least || *abort_flag) return;
+                    if ((spin & 1023u) == 0) {
+                        const uint64_t now = global_timer_ns();
+                        if (t0 == 0) t0 = now;
+                        else if (now - t0 > 2000000000ull) {
+                            *abort_flag = 1;
+                            return;
                         }
                     }
                 }
-                group_sync(bar_id);
-            }
-            const bool tail = pos0 + kTilePos > L - gamma;
-            const int gmin = pos - L + gamma;           // tail index of `pos`: queries below it do not see it
-            uint8_t *prow = gbase + sm.p + pb * (NP * 256) + row * 16;
-            uint4 pk[kMaxChunks];   // this position's probabilities, 8 columns per entry
+            };
+            // buffers of this group's tile advance by counting, not by dividing
+            int sbi = grp % cfg.sb, pb = grp % cfg.pb;
+            auto advance = [](int &idx, int n) {
+                idx += kSoftmaxGroups;
+                while (idx >= n) idx -= n;
+            };
+            for (int i = grp; i < T; i += kSoftmaxGroups) {
+                const int pos0 = (t_begin + i) * kTilePos;
+                const int pos = pos0 + row;
+                if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 0);     // starts waiting for S^T
+                mbar_wait(s_full(i), hand_parity(i), abort_flag);
+                if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 1);     // S^T there
+                tc_fence_after();
+                const uint32_t s_addr = tm_s0 + sbi * NP + lane_addr;
+                // The oldest uncommitted tile is the one whose group may move m.  Tile 0 is that
+                // from the start and sets m up; the others read m under an epoch and check it
+                // when their turn comes.
+                bool my_turn = i == 0;
+                uint32_t e0 = 0;
+                if (i == 0) {
+                    if (!kFp8) {
+                        // reference exponent of each row: its score at the split's first position
+                        // (every warp reads the chunks c8 = its quarter, quarter + 4, ... from the TMEM
+                        // lanes it can reach; only the first quarter holds position 0)
+                        if (wq == 0) {
+#pragma unroll 1
+                            for (int cb = 0; cb < n8; cb += 2) {
+                                uint32_t r[2][8];
+#pragma unroll
+                                for (int u = 0; u < 2; ++u)
+                                    if (cb + u < n8) tmem_ld_x8(s_addr + (cb + u) * 8, r[u]);
+                                tmem_wait_ld();
+                                if (lane == 0) {
+#pragma unroll
+                                    for (int u = 0; u < 2; ++u)
+                                        if (cb + u < n8) {
+#pragma unroll
+                                            for (int k = 0; k < 8; ++k)
+                                                m_s[(cb + u) * 8 + k] = __uint_as_float(r[u][k]) * scale - kLift;
+                                        }
+                                }
+                            }
+                        }
+                        group_sync(bar_id);
+                        if (gtid == 0) {
+                            __threadfence_block();
+                            *epoch_s = 1;
+                        }
+                    }
+                } else {
+                    if (i < kSoftmaxGroups) wait_counter(epoch_s, 1);     // m comes from the first tile
+                    e0 = *epoch_s;
+                    __threadfence_block();
+                }
+                const bool tail = pos0 + kTilePos > L - gamma;
+                const int gmin = pos - L + gamma;           // tail index of `pos`: queries below it do not see it
+                // P^T goes straight to shared memory: the P.V product that read this buffer last is done
+                // (tile i - pb; this group saw tile i - 3 - pb's product done a turn ago)
+                if (i >= cfg.pb) mbar_wait(p_free(i - cfg.pb), hand_parity(i - cfg.pb), abort_flag);
+                if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 2);     // P buffer free
+                uint8_t *prow = gbase + sm.p + pb * (NP * 256) + row * 16;
 
-            for (int attempt = 0; attempt < 3; ++attempt) {
                 // fp8 cache: E4M3 has 17 binades, so the reference exponent of a row starts
                 // from the largest score of the split's first tile (the path below), not
                 // from whatever score its first position happens to have
-                const bool first_max = kFp8 && i == 0 && attempt == 0;
-                if (!first_max) {
-                    const float gmax =
-                        !tail ? softmax_pass<0, kFp8>(s_addr, c_lo, c_hi, m_s, scale, vis_s, G, gmin, pk)
-                              : softmax_pass<kTree ? 2 : 1, kFp8>(s_addr, c_lo, c_hi, m_s, scale, vis_s, G, gmin, pk);
-                    if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 2);     // exponentials done
-                    if (!group_any(bar_id, gmax > kLimit)) break;
-                }
+                bool take_max = kFp8 && i == 0;
+                for (int attempt = 0; attempt < 4; ++attempt) {
+                    float gmax = -INFINITY;
+                    if (!take_max)
+                        gmax = !tail ? softmax_pass<0, kFp8>(s_addr, n8, m_s, scale, vis_s, G, gmin, prow,
+                                                             warp == kSoftmaxWarp0 ? tile_tr : nullptr, i)
+                                     : softmax_pass<kTree ? 2 : 1, kFp8>(s_addr, n8, m_s, scale, vis_s, G, gmin, prow, nullptr, i);
+                    if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 3);     // exponentials done
+                    if (!my_turn) {
+                        wait_counter(committed_s, (uint32_t)i);
+                        my_turn = true;
+                        __threadfence_block();
+                        const uint32_t e1 = *epoch_s;       // final: only this group can move m now
+                        const bool stale = e1 != e0;
+                        if (!group_any(bar_id, stale || gmax > kLimit)) break;
+                        // m moved while some thread computed under the old one: once more
+                        if (group_any(bar_id, stale)) continue;
+                    } else if (!take_max && !group_any(bar_id, gmax > kLimit)) {
+                        break;
+                    }
+                    take_max = false;
 
-                // ---- a score ran past the guard: move m up to the tile maximum ----
-                for (int c8 = c_lo; c8 < c_hi; ++c8) {
-                    uint32_t r[8];
-                    tmem_ld_x8(s_addr + c8 * 8, r);
-                    tmem_wait_ld();
+                    // ---- a score ran past the guard: move m up to the tile maximum ----
+                    // (the masked form, with its divisions, only where the tile reaches the draft slots)
+                    auto tile_max = [&](auto masked) {
+#pragma unroll 1
+                        for (int c8 = 0; c8 < n8; ++c8) {
+                            uint32_t r[8];
+                            tmem_ld_x8(s_addr + c8 * 8, r);
+                            tmem_wait_ld();
+                            // eight reductions in flight, then their results stored
+                            float s2[8];
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        float s2 = __uint_as_float(r[k]) * scale;
-                        if (tail && (kTree ? !column_sees(vis_s[c8 * 8 + k], gmin) : (c8 * 8 + k) / G < gmin))
-                            s2 = -INFINITY;
-                        s2 = warp_max_f32(s2);
-                        if (lane == 0) tmx_s[wq * NP + c8 * 8 + k] = s2;
-                    }
-                }
-                group_sync(bar_id);
-                for (int n = c_lo * 8 + gtid; n < c_hi * 8; n += 128) {
-                    const float mt = fmaxf(fmaxf(tmx_s[n], tmx_s[NP + n]),
-                                           fmaxf(tmx_s[2 * NP + n], tmx_s[3 * NP + n])) - kLift;
-                    const float mo = m_s[n];
-                    const float mn = fmaxf(mo, mt);
-                    dl_s[n] = mo - mn;              // <= 0
-                    m_s[n] = mn;
-                }
-                group_sync(bar_id);
-                if (i > 0) {
-                    // O^T and the sums were accumulated under the old m: rescale this
-                    // group's columns once PV(i-1) has finished
-                    {
-                        // the P buffer of tile i - 1 and the round it was filled in
-                        const int pp = pb == 0 ? cfg.pb - 1 : pb - 1;
-                        const uint32_t pr = pb == 0 ? pb_round - 1 : pb_round;
-                        mbar_wait(p_free(pp), pr & 1, abort_flag);
-                    }
-                    tc_fence_after();
-                    // (fp8 cache: accumulator columns 2n and 2n + 1 belong to row n)
-                    for (int c = c_lo * kAccCols; c < c_hi * kAccCols; ++c) {
-                        uint32_t r[8];
-                        tmem_ld_x8(tm_o + lane_addr + c * 8, r);
-                        tmem_wait_ld();
+                            for (int k = 0; k < 8; ++k) {
+                                s2[k] = __uint_as_float(r[k]) * scale;
+                                if constexpr (decltype(masked)::value) {
+                                    if (kTree ? !column_sees(vis_s[c8 * 8 + k], gmin) : (c8 * 8 + k) / G < gmin)
+                                        s2[k] = -INFINITY;
+                                }
+                            }
 #pragma unroll
-                        for (int k = 0; k < 8; ++k)
-                            r[k] = __float_as_uint(__uint_as_float(r[k]) * ex2(dl_s[(c * 8 + k) / kAccCols]));
-                        tmem_st_x8(tm_o + lane_addr + c * 8, r);
-                        if (wq == 0) {
-                            tmem_ld_x8(tm_l + c * 8, r);
+                            for (int k = 0; k < 8; ++k) s2[k] = warp_max_f32(s2[k]);
+                            if (lane == 0) {
+                                float *dst = tmx_s + wq * NP + c8 * 8;
+                                *reinterpret_cast<float4 *>(dst) = make_float4(s2[0], s2[1], s2[2], s2[3]);
+                                *reinterpret_cast<float4 *>(dst + 4) = make_float4(s2[4], s2[5], s2[6], s2[7]);
+                            }
+                        }
+                    };
+                    if (tail) tile_max(std::true_type{});
+                    else tile_max(std::false_type{});
+                    group_sync(bar_id);
+                    for (int n = gtid; n < n8 * 8; n += 128) {
+                        const float mt = fmaxf(fmaxf(tmx_s[n], tmx_s[NP + n]),
+                                               fmaxf(tmx_s[2 * NP + n], tmx_s[3 * NP + n])) - kLift;
+                        const float mo = m_s[n];
+                        const float mn = fmaxf(mo, mt);
+                        dl_s[n] = mo - mn;              // <= 0
+                        m_s[n] = mn;
+                    }
+                    group_sync(bar_id);
+                    if (gtid == 0) {
+                        __threadfence_block();
+                        *epoch_s = *epoch_s + 1;
+                    }
+                    if (i > 0) {
+                        // O^T and the sums were accumulated under the old m: rescale them once
+                        // the P.V product of tile i - 1 has finished (tile i - 1 is committed, so
+                        // its group has seen the product of tile i - 4 or a later one done)
+                        mbar_wait(p_free(i - 1), hand_parity(i - 1), abort_flag);
+                        tc_fence_after();
+                        // (fp8 cache: accumulator columns 2n and 2n + 1 belong to row n)
+                        for (int c = 0; c < n8 * kAccCols; ++c) {
+                            uint32_t r[8];
+                            tmem_ld_x8(tm_o + lane_addr + c * 8, r);
                             tmem_wait_ld();
 #pragma unroll
                             for (int k = 0; k < 8; ++k)
                                 r[k] = __float_as_uint(__uint_as_float(r[k]) * ex2(dl_s[(c * 8 + k) / kAccCols]));
-                            tmem_st_x8(tm_l + c * 8, r);
+                            tmem_st_x8(tm_o + lane_addr + c * 8, r);
+                            if (wq == 0) {
+                                tmem_ld_x8(tm_l + c * 8, r);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int k = 0; k < 8; ++k)
+                                    r[k] = __float_as_uint(__uint_as_float(r[k]) * ex2(dl_s[(c * 8 + k) / kAccCols]));
+                                tmem_st_x8(tm_l + c * 8, r);
+                            }
+                        }
+                        tmem_wait_st();
+                        tc_fence_before();
+                    }
+                    group_sync(bar_id);
+                }
+                if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 4);     // this tile's turn came and m stood
+                // m stands for this tile: the next tile's group may take its turn
+                if (gtid == 0) {
+                    __threadfence_block();
+                    *committed_s = (uint32_t)i + 1;
+                }
+                if (pos0 + kTilePos > L) {
+                    // slots at or beyond kv_len hold whatever the cache holds: zero their V
+                    // rows so that 0 * junk cannot poison the accumulators.  Once the product of
+                    // tile i - 1 is done, the V slot's barrier can only be in this tile's phase.
+                    if (i > 0) mbar_wait(p_free(i - 1), hand_parity(i - 1), abort_flag);
+                    const int vsl = i % cfg.vs;
+                    mbar_wait(v_full(vsl), (i / cfg.vs) & 1, abort_flag);
+                    if (pos >= L) {
+                        uint8_t *vrow = gbase + sm.v + vsl * kSlot + row * 128;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            *reinterpret_cast<uint4 *>(vrow + c * 16) = make_uint4(0, 0, 0, 0);
+                            if (!kFp8) *reinterpret_cast<uint4 *>(vrow + kBoxBytes + c * 16) = make_uint4(0, 0, 0, 0);
                         }
                     }
-                    tmem_wait_st();
-                    tc_fence_before();
                 }
-                group_sync(bar_id);
+                // one arrival per warp: S^T has been read (the K.Q^T of a later tile may overwrite
+                // it) and P^T, with any zeroed V rows, is in shared memory
+                tc_fence_before();
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(s_free(i));
+                    mbar_arrive(p_full(i));
+                }
+                if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 5);     // P^T handed over
+                advance(sbi, cfg.sb);
+                advance(pb, cfg.pb);
             }
-            if (tail && grp == 0) {
-                // slots at or beyond kv_len hold whatever the cache holds: zero their V
-                // rows so that 0 * junk cannot poison the accumulators
-                mbar_wait(v_full(vsl), vs_round & 1, abort_flag);
-                if (pos >= L) {
-                    uint8_t *vrow = gbase + sm.v + vsl * kSlot + row * 128;
+        } else {
+            // ring positions advance by counting, not by dividing
+            int pb = 0, vsl = 0;                 // P buffer and V slot of tile i
+            uint32_t pb_round = 0, vs_round = 0; // how often each ring has wrapped
+            for (int i = 0; i < T; ++i) {
+                const int pos0 = (t_begin + i) * kTilePos;
+                const int pos = pos0 + row;
+                const int sb = i & 1;
+                if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 0);     // starts waiting for S^T
+                mbar_wait(s_full(i), hand_parity(i), abort_flag);
+                if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 1);     // S^T there
+                tc_fence_after();
+                const uint32_t s_addr = tm_s0 + sb * NP + lane_addr;
+                if (!kFp8 && i == 0) {
+                    // reference exponent of each row: its score at the split's first position
+                    if (wq == 0) {
+                        for (int c8 = c_lo; c8 < c_hi; ++c8) {
+                            uint32_t r[8];
+                            tmem_ld_x8(s_addr + c8 * 8, r);
+                            tmem_wait_ld();
+                            if (lane == 0) {
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        *reinterpret_cast<uint4 *>(vrow + c * 16) = make_uint4(0, 0, 0, 0);
-                        if (!kFp8) *reinterpret_cast<uint4 *>(vrow + kBoxBytes + c * 16) = make_uint4(0, 0, 0, 0);
+                                for (int k = 0; k < 8; ++k) m_s[c8 * 8 + k] = __uint_as_float(r[k]) * scale - kLift;
+                            }
+                        }
+                    }
+                    group_sync(bar_id);
+                }
+                const bool tail = pos0 + kTilePos > L - gamma;
+                const int gmin = pos - L + gamma;           // tail index of `pos`: queries below it do not see it
+                uint8_t *prow = gbase + sm.p + pb * (NP * 256) + row * 16;
+                uint4 pk[kMaxChunks];   // this position's probabilities, 8 columns per entry
+
+                for (int attempt = 0; attempt < 3; ++attempt) {
+                    // fp8 cache: E4M3 has 17 binades, so the reference exponent of a row starts
+                    // from the largest score of the split's first tile (the path below), not
+                    // from whatever score its first position happens to have
+                    const bool first_max = kFp8 && i == 0 && attempt == 0;
+                    if (!first_max) {
+                        const float gmax =
+                            !tail ? softmax_pass_share<0, kFp8>(s_addr, c_lo, c_hi, m_s, scale, vis_s, G, gmin, pk)
+                                  : softmax_pass_share<kTree ? 2 : 1, kFp8>(s_addr, c_lo, c_hi, m_s, scale, vis_s, G, gmin, pk);
+                        if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 2);     // exponentials done
+                        if (!group_any(bar_id, gmax > kLimit)) break;
+                    }
+
+                    // ---- a score ran past the guard: move m up to the tile maximum ----
+                    for (int c8 = c_lo; c8 < c_hi; ++c8) {
+                        uint32_t r[8];
+                        tmem_ld_x8(s_addr + c8 * 8, r);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            float s2 = __uint_as_float(r[k]) * scale;
+                            if (tail && (kTree ? !column_sees(vis_s[c8 * 8 + k], gmin) : (c8 * 8 + k) / G < gmin))
+                                s2 = -INFINITY;
+                            s2 = warp_max_f32(s2);
+                            if (lane == 0) tmx_s[wq * NP + c8 * 8 + k] = s2;
+                        }
+                    }
+                    group_sync(bar_id);
+                    for (int n = c_lo * 8 + gtid; n < c_hi * 8; n += 128) {
+                        const float mt = fmaxf(fmaxf(tmx_s[n], tmx_s[NP + n]),
+                                               fmaxf(tmx_s[2 * NP + n], tmx_s[3 * NP + n])) - kLift;
+                        const float mo = m_s[n];
+                        const float mn = fmaxf(mo, mt);
+                        dl_s[n] = mo - mn;              // <= 0
+                        m_s[n] = mn;
+                    }
+                    group_sync(bar_id);
+                    if (i > 0) {
+                        // O^T and the sums were accumulated under the old m: rescale this
+                        // group's columns once PV(i-1) has finished
+                        mbar_wait(p_free(i - 1), hand_parity(i - 1), abort_flag);
+                        tc_fence_after();
+                        // (fp8 cache: accumulator columns 2n and 2n + 1 belong to row n)
+                        for (int c = c_lo * kAccCols; c < c_hi * kAccCols; ++c) {
+                            uint32_t r[8];
+                            tmem_ld_x8(tm_o + lane_addr + c * 8, r);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int k = 0; k < 8; ++k)
+                                r[k] = __float_as_uint(__uint_as_float(r[k]) * ex2(dl_s[(c * 8 + k) / kAccCols]));
+                            tmem_st_x8(tm_o + lane_addr + c * 8, r);
+                            if (wq == 0) {
+                                tmem_ld_x8(tm_l + c * 8, r);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int k = 0; k < 8; ++k)
+                                    r[k] = __float_as_uint(__uint_as_float(r[k]) * ex2(dl_s[(c * 8 + k) / kAccCols]));
+                                tmem_st_x8(tm_l + c * 8, r);
+                            }
+                        }
+                        tmem_wait_st();
+                        tc_fence_before();
+                    }
+                    group_sync(bar_id);
+                }
+                if (tail && grp == 0) {
+                    // slots at or beyond kv_len hold whatever the cache holds: zero their V
+                    // rows so that 0 * junk cannot poison the accumulators
+                    mbar_wait(v_full(vsl), vs_round & 1, abort_flag);
+                    if (pos >= L) {
+                        uint8_t *vrow = gbase + sm.v + vsl * kSlot + row * 128;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            *reinterpret_cast<uint4 *>(vrow + c * 16) = make_uint4(0, 0, 0, 0);
+                            if (!kFp8) *reinterpret_cast<uint4 *>(vrow + kBoxBytes + c * 16) = make_uint4(0, 0, 0, 0);
+                        }
                     }
                 }
-            }
-            if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 3);     // the group agrees: no rescale
-            // P^T goes to shared memory once the P.V product that read this buffer is done
-            if (pb_round > 0) mbar_wait(p_free(pb), (pb_round - 1) & 1, abort_flag);
-            if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 4);     // P buffer free
+                if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 3);     // the group agrees: no rescale
+                // P^T goes to shared memory once the P.V product that read this buffer is done
+                if (i >= cfg.pb) mbar_wait(p_free(i - cfg.pb), hand_parity(i - cfg.pb), abort_flag);
+                if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 4);     // P buffer free
 #pragma unroll
-            for (int j = 0; j < kMaxChunks; ++j)
-                if (c_lo + j < c_hi) *reinterpret_cast<uint4 *>(prow + (c_lo + j) * 2048) = pk[j];
-            // one arrival per warp: S^T has been read (the next K.Q^T but one may overwrite
-            // it) and P^T, with any zeroed V rows, is in shared memory
-            tc_fence_before();
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(s_free(sb));
-                mbar_arrive(p_full(pb));
+                for (int j = 0; j < kMaxChunks; ++j)
+                    if (c_lo + j < c_hi) *reinterpret_cast<uint4 *>(prow + (c_lo + j) * 2048) = pk[j];
+                // one arrival per warp: S^T has been read (the next K.Q^T but one may overwrite
+                // it) and P^T, with any zeroed V rows, is in shared memory
+                tc_fence_before();
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(s_free(i));
+                    mbar_arrive(p_full(i));
+                }
+                if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 5);     // P^T stored and handed over
+                if (++pb == cfg.pb) { pb = 0; ++pb_round; }
+                if (++vsl == cfg.vs) { vsl = 0; ++vs_round; }
             }
-            if (warp == kSoftmaxWarp0) LVSPEC_TILE_TS(tile_tr, 0, i, 5);     // P^T stored and handed over
-            if (++pb == cfg.pb) { pb = 0; ++pb_round; }
-            if (++vsl == cfg.vs) { vsl = 0; ++vs_round; }
         }
 
         // ---------------------------------------------------------------- epilogue
-        {
-            const int pp = pb == 0 ? cfg.pb - 1 : pb - 1;
-            const uint32_t pr = pb == 0 ? pb_round - 1 : pb_round;
-            mbar_wait(p_free(pp), pr & 1, abort_flag);
-        }
+        // (every group takes its share of the columns)
+        // the last P.V product has finished (and with it all before)
+        mbar_wait(pv_done, 0, abort_flag);
         tc_fence_after();
         if (p.n_split == 1) {
             // a single split: nothing to merge, normalise and write the results here
@@ -1039,28 +1356,49 @@ bool make_q_map(CUtensorMap *map, const void *ptr, int B, int gamma, int Hq, int
 
 constexpr uint32_t kMaxSmem = 232448 - 1024;   // 227 KB less the alignment slack
 
-TcConfig pick_config(int M, int page_slots, bool fp8)
+TcConfig pick_config(int M, int page_slots, bool fp8, bool turns)
 {
     TcConfig c;
     c.n_pad = (M + 15) & ~15;
     c.page_slots = page_slots;
     c.slot_bytes = fp8 ? kBoxBytes : kSlotBytes;
-    // Six ring slots when they fit, also at the price of the second P buffer (with 40 rows
-    // the stream is bound by HBM: bytes in flight count, and the probabilities wait in
-    // registers for the buffer anyway); below that, a second P buffer before a fifth slot
-    // (with 80 rows the chain softmax -> P.V -> next softmax bounds the tile, and two
-    // buffers with 2 + 2 slots beat one with 2 + 3).  An fp8 tile is half the bytes: twice
-    // the slots for the same bytes in flight.
-    const int tries[6][3] = {{3, 3, 2}, {3, 3, 1}, {2, 3, 2}, {2, 2, 2}, {2, 3, 1}, {2, 2, 1}};
-    const int tries8[6][3] = {{5, 6, 2}, {5, 5, 2}, {4, 5, 2}, {4, 4, 2}, {4, 4, 1}, {3, 3, 1}};
-    for (int t = 0; t < 6; ++t) {
-        const int *tr = fp8 ? tries8[t] : tries[t];
-        c.ks = tr[0]; c.vs = tr[1]; c.pb = tr[2];
-        if (smem_map(c).total <= kMaxSmem) break;
+    const int acc = fp8 ? 4 : 2;     // TMEM columns per padded row of O^T and the sums
+    if (!turns) {
+        // All groups on every tile: S^T twice.  Six ring slots when they fit, also at the
+        // price of the second P buffer (with 40 rows the stream is bound by HBM: bytes in
+        // flight count, and the probabilities wait in registers for the buffer anyway).
+        c.sb = 2;
+        const int tries[6][3] = {{3, 3, 2}, {3, 3, 1}, {2, 3, 2}, {2, 2, 2}, {2, 3, 1}, {2, 2, 1}};
+        for (int t = 0; t < 6; ++t) {
+            c.ks = tries[t][0]; c.vs = tries[t][1]; c.pb = tries[t][2];
+            if (smem_map(c).total <= kMaxSmem) break;
+        }
+    } else {
+        // Tiles in turn: an S^T buffer per softmax group when TMEM has the columns, else
+        // two.  Shared memory: a P^T buffer per group before more ring slots (a group that
+        // shares its buffer waits for the product of an earlier tile before it can store
+        // anything); of the rings, V slots are held longer than K slots.  An fp8 tile is
+        // half the bytes: twice the slots for the same bytes in flight.
+        c.sb = (kSoftmaxGroups + acc) * c.n_pad <= 512 ? kSoftmaxGroups : 2;
+        const int tries[8][3] = {{3, 3, 3}, {2, 3, 3}, {3, 2, 3}, {2, 2, 3}, {2, 2, 2}, {2, 2, 1}, {1, 2, 1}, {1, 1, 1}};
+        const int tries8[8][3] = {{5, 6, 3}, {5, 5, 3}, {4, 5, 3}, {4, 4, 3}, {4, 4, 2}, {3, 3, 2}, {3, 3, 1}, {2, 2, 1}};
+        for (int t = 0; t < 8; ++t) {
+            const int *tr = fp8 ? tries8[t] : tries[t];
+            c.ks = tr[0]; c.vs = tr[1]; c.pb = tr[2];
+            if (smem_map(c).total <= kMaxSmem) break;
+        }
     }
-    // S^T twice, O^T and the sums: 4 columns per padded row, 6 with an fp8 cache
+    // LVSPEC_TC_RING="K slots,V slots,P buffers,S buffers" overrides the choice (for
+    // measurements; a combination that does not fit is refused by the launch)
+    if (const char *e = std::getenv("LVSPEC_TC_RING")) {
+        int ks, vs, pb, sb;
+        if (std::sscanf(e, "%d,%d,%d,%d", &ks, &vs, &pb, &sb) == 4 && ks >= 1 && ks <= 8 && vs >= 1 && vs <= 8 &&
+            pb >= 1 && pb <= kSoftmaxGroups && sb >= 2 && sb <= kSoftmaxGroups && (turns || (sb == 2 && pb <= 2))) {
+            c.ks = ks; c.vs = vs; c.pb = pb; c.sb = sb;
+        }
+    }
     int cols = 32;
-    while (cols < (fp8 ? 6 : 4) * c.n_pad) cols <<= 1;
+    while (cols < (c.sb + acc) * c.n_pad) cols <<= 1;
     c.tmem_cols = cols;
     return c;
 }
@@ -1081,7 +1419,16 @@ cudaError_t launch_attn_tc(const AttnParams &p, const SeqInfo &seq, cudaStream_t
     // paged: one block-table entry per tile of the longest split, rounded up to 4
     const int tiles = (p.Lmax + kTilePos - 1) / kTilePos;
     const bool fp8 = p.fp8 != 0;
-    P.cfg = pick_config(p.M, paged ? ((tiles + p.n_split - 1) / p.n_split + 4) & ~3 : 0, fp8);
+    // Tiles in turn where a CTA streams long enough for the throughput of the softmax stage
+    // to outweigh its latency at the two ends of the stream (measured on the 40/8-head sweep:
+    // 5 to 10 % faster from about a hundred tiles per CTA, slower below 32), and with an fp8
+    // cache of up to 64 padded rows (half the bytes per tile for the same work; with more
+    // rows TMEM holds only two S^T buffers and the shared columns win).
+    // LVSPEC_TC_TURNS=0/1 overrides the choice (for measurements).
+    bool turns = (tiles + p.n_split - 1) / p.n_split >= 96 || (fp8 && p.M <= 64);
+    if (const char *e = std::getenv("LVSPEC_TC_TURNS"))
+        if (e[0] == '0' || e[0] == '1') turns = e[0] == '1';
+    P.cfg = pick_config(p.M, paged ? ((tiles + p.n_split - 1) / p.n_split + 4) & ~3 : 0, fp8, turns);
     if (smem_map(P.cfg).total > kMaxSmem || P.cfg.tmem_cols > 512) return cudaErrorInvalidConfiguration;
     CUtensorMap mk, mv, mq;
     const int map_len = paged ? p.page_size : p.Lmax;
@@ -1094,9 +1441,13 @@ cudaError_t launch_attn_tc(const AttnParams &p, const SeqInfo &seq, cudaStream_t
     const size_t smem = smem_map(P.cfg).total + 1024;
     const bool tree = p.branch_len != p.gamma;
     if ((tree && paged) || (fp8 && (tree || paged))) return cudaErrorNotSupported;
-    auto kernel = fp8 ? attn_tc_kernel<false, false, true>
-                      : (paged ? attn_tc_kernel<false, true, false>
-                               : (tree ? attn_tc_kernel<true, false, false> : attn_tc_kernel<false, false, false>));
+    auto kernel = fp8 ? (turns ? attn_tc_kernel<false, false, true, true> : attn_tc_kernel<false, false, true, false>)
+                  : turns ? (paged ? attn_tc_kernel<false, true, false, true>
+                                   : (tree ? attn_tc_kernel<true, false, false, true>
+                                           : attn_tc_kernel<false, false, false, true>))
+                          : (paged ? attn_tc_kernel<false, true, false, false>
+                                   : (tree ? attn_tc_kernel<true, false, false, false>
+                                           : attn_tc_kernel<false, false, false, false>));
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};

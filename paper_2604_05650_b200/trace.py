@@ -80,7 +80,7 @@ def main() -> None:
     shape = binding.attn_shape(B, g, Hq, Hkv, D, L, args.n_split, binding.KERNEL_TCGEN05)
     kv_len = np.full((B,), L, np.int32)
     span = np.tile(np.asarray([cfg.span], np.int32), (B, 1))
-    words = torch.zeros(8 + 8 * CTA_RECORDS + 3 * 32 * 8, dtype=torch.int64, device=dev)
+    words = torch.zeros(8 + 8 * CTA_RECORDS + 4 * 32 * 8, dtype=torch.int64, device=dev)
     stream = torch.cuda.Stream()
 
     def calls():
@@ -120,20 +120,24 @@ def main() -> None:
         if len(A):
             print(f"layer {l} attention ({len(A)} CTAs): resident {three(A[:, 3])} | past the prologue {three(A[:, 4])}"
                   f" | last K.Q^T done {three(A[:, 5])} | end {three(A[:, 6])}")
+            late = A[np.argsort(A[:, 6])[-4:]]
+            print("        last to finish (split, KV head: end, tiles done at): " + "; ".join(
+                f"{int(r[2]) % 1000}, {int(r[2]) // 1000 % 1000}: {us(r[6])}, {us(r[5])}" for r in late))
         if len(C):
             print(f"        merge ({len(C)} CTAs): resident {three(C[:, 3])} | attention grid complete {three(C[:, 4])}"
                   f" | end {three(C[:, 6])}")
-    T = w[8 + 8 * CTA_RECORDS:].reshape(3, 32, 8)
+    T = w[8 + 8 * CTA_RECORDS:].reshape(4, 32, 8)
     if T.any():
         c0 = int(T[T > 0].min())
         print("tiles of attention CTA (split 3, KV head 2) of the last traced layer; cycles from its first stamp")
-        print("tile | K.Q^T issuer: waits for K, K there, S^T free, issued | softmax warp: waits for S^T, there, exponentials done,"
-              " group agreed, P buffer free, P^T handed over | P.V issuer: waits for P^T, there, V there, issued")
+        print("tile | K.Q^T issuer: waits for K, K there, S^T free, issued | first softmax warp (it takes every third tile): waits"
+              " for S^T, there, P buffer free, exponentials done, its turn came and m stood, P^T handed over | P.V issuer: waits"
+              " for P^T, there, V there, issued | softmax pass, per four chunks of columns: asks for S^T, has it, probabilities stored")
         rel = lambda a: " ".join(f"{int(x) - c0:6d}" if x else "     -" for x in a)
         for i in range(32):
             if not T[:, i].any():
                 break
-            print(f"{i:3d} | {rel(T[1, i, :4])} | {rel(T[0, i, :6])} | {rel(T[2, i, :4])}")
+            print(f"{i:3d} | {rel(T[1, i, :4])} | {rel(T[0, i, :6])} | {rel(T[2, i, :4])} | {rel(T[3, i, :6])}")
     ctx.close()
 
 
