@@ -199,8 +199,13 @@ cos_tc_kernel(const CosParams P, const __grid_constant__ CUtensorMap tmap_v,
             const uint64_t stream_policy = l2_evict_first_policy();
             int n = 0;                       // stages filled so far
             bool ok = true;
+            // Every CTA walks the channels from a different slab on (and around): at a row
+            // pitch like 10 KB the same slab of all rows shares its low address bits, and
+            // with all CTAs on the same slab the requests crowd on few memory channels.
+            const int kc0 = (int)((blockIdx.x * 37u) % (unsigned)KC);
             while (ok && walk.next()) {
-                for (int kc = 0; kc < KC; ++kc, ++n) {
+                for (int kci = 0; kci < KC; ++kci, ++n) {
+                    const int kc = kci + kc0 < KC ? kci + kc0 : kci + kc0 - KC;
                     const int s = n % S;
                     if (n >= S && !mbar_wait(empty(s), ((n / S) - 1) & 1, abort_flag)) { ok = false; break; }
                     const uint32_t dst = base + s * stage_bytes;
@@ -402,6 +407,7 @@ constexpr int kTopThreads = 1024;
 
 constexpr int kTopPerThread = 32;      // fast path: lv <= 32 * 1024
 constexpr int kTopCandidates = 2048;
+constexpr int kRankCandidates = 256;    // up to here the candidates are ranked by counting, not sorted
 
 // descending bitonic sort of a power-of-two array of keys in shared memory
 __device__ void bitonic_sort_desc(uint32_t *a, int n, int tid)
@@ -435,6 +441,7 @@ __global__ void __launch_bounds__(kTopThreads) topn_mean_kernel(const RelevanceP
     asm volatile("griddepcontrol.wait;" ::: "memory");
     __shared__ uint32_t keys[kTopCandidates];
     __shared__ uint32_t hist[256];
+    __shared__ uint32_t ranked[kRankCandidates];
     __shared__ uint32_t sel_prefix, sel_need, n_cand;
     __shared__ float warp_sum[kTopThreads / 32];
     __shared__ int n_values;
@@ -511,6 +518,27 @@ __global__ void __launch_bounds__(kTopThreads) topn_mean_kernel(const RelevanceP
         }
         __syncthreads();
         const uint32_t c = n_cand;
+        if (c <= (uint32_t)kRankCandidates) {
+            // few candidates (the usual case): every candidate counts those ahead of it
+            // (larger key, or equal key and lower index) and the first n go to their places;
+            // one pass and one barrier where a block-wide sort takes dozens
+            for (uint32_t i = tid; i < c; i += kTopThreads) {
+                const uint32_t key = keys[i];
+                uint32_t rank = 0;
+                for (uint32_t j = 0; j < c; ++j) {
+                    const uint32_t kj = keys[j];
+                    rank += (kj > key || (kj == key && j < i)) ? 1u : 0u;
+                }
+                if (rank < n) ranked[rank] = key;
+            }
+            __syncthreads();
+            if (tid == 0) {
+                float sum = 0.f;
+                for (uint32_t i = 0; i < n; ++i) sum += key_float(ranked[i]);
+                *out = sum / (float)n;
+            }
+            return;
+        }
         if (c <= (uint32_t)kTopCandidates) {
             int pow2 = 32;
             while ((uint32_t)pow2 < c) pow2 <<= 1;
