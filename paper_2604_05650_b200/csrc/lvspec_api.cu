@@ -94,11 +94,11 @@ lvspec_status_t ensure(lvspec_ctx *ctx, void **buf, size_t *have, size_t want, b
     return LVSPEC_OK;
 }
 
-// The tensor-core kernel covers head_dim 128 with at least one full tile of
+// The tensor-core kernel covers head_dim 64 and 128 with at least one full tile of
 // cache; everything else runs on the CUDA-core kernel.
 bool tc_shape(const lvspec_attn_shape_t *s)
 {
-    return s->head_dim == 128 && s->kv_capacity >= 128;
+    return (s->head_dim == 128 || s->head_dim == 64) && s->kv_capacity >= 128;
 }
 
 int resolve_kernel(const lvspec_attn_shape_t *s)
@@ -304,7 +304,7 @@ lvspec_status_t run_attention(lvspec_ctx *ctx, const lvspec_attn_shape_t *s, con
             return fail(ctx, LVSPEC_ERR_UNSUPPORTED,
                         p.fp8 ? "the fp8 cache needs head_dim 128, kv_capacity >= 128 and at most 80 query rows "
                                 "per KV head"
-                              : "the tcgen05 kernel needs head_dim 128 and kv_capacity >= 128");
+                              : "the tcgen05 kernel needs head_dim 64 or 128 and kv_capacity >= 128");
         e = launch_attn_tc(p, seq, ctx->stream, &launches);
     } else {
         e = launch_attn_simt(p, seq, ctx->stream, &launches);

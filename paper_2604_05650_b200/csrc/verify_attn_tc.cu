@@ -335,7 +335,11 @@ __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUtensorMap tmap_k,
                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_q)
 {
-    constexpr uint32_t kSlot = kFp8 ? kBoxBytes : kSlotBytes;   // bytes of one K or V tile
+    // bytes of one K or V tile: two 64-channel boxes at head_dim 128 (bf16), one box at
+    // head_dim 64 and for an fp8 tile of 128 channels
+    const uint32_t kSlot = (uint32_t)P.cfg.slot_bytes;
+    const bool two_boxes = kSlot == kSlotBytes;
+    const int D = P.a.D;
     extern __shared__ uint8_t smem_raw[];
     const AttnParams &p = P.a;
     const TcConfig cfg = P.cfg;
@@ -378,7 +382,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
     const int T = t_base + (split < t_rem ? 1 : 0);
 
     const size_t unit = ((size_t)b * p.Hkv + kvh) * p.n_split + split;
-    float *part_o = p.part_o + unit * (size_t)M * 128;
+    float *part_o = p.part_o + unit * (size_t)M * P.a.D;
     float *part_stat = p.part_stat + unit * (size_t)M * 4;
     if (T <= 0) {   // a split with no tile: contributes nothing
         if (tid == 0) {
@@ -446,7 +450,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         tile_at(i, pos0, map_row);
         mbar_arrive_expect_tx(k_full(ks), kSlot);
         tma_load_4d_hint(base + sm.k + ks * kSlot, &tmap_k, k_full(ks), 0, pos0, kvh, map_row, stream_policy);
-        if (!kFp8)
+        if (two_boxes)
             tma_load_4d_hint(base + sm.k + ks * kSlot + kBoxBytes, &tmap_k, k_full(ks), 64, pos0, kvh, map_row,
                              stream_policy);
     };
@@ -456,7 +460,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
         tile_at(i, pos0, map_row);
         mbar_arrive_expect_tx(v_full(vsl), kSlot);
         tma_load_4d_hint(base + sm.v + vsl * kSlot, &tmap_v, v_full(vsl), 0, pos0, kvh, map_row, stream_policy);
-        if (!kFp8)
+        if (two_boxes)
             tma_load_4d_hint(base + sm.v + vsl * kSlot + kBoxBytes, &tmap_v, v_full(vsl), 64, pos0, kvh, map_row,
                              stream_policy);
     };
@@ -506,9 +510,9 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             first_v = min(T, cfg.vs);
             load_k(0);
             if (!kFp8) {
-                mbar_arrive_expect_tx(q_full, (uint32_t)M * 256u);
+                mbar_arrive_expect_tx(q_full, (uint32_t)(M * D) * 2u);
                 tma_load_4d(base + sm.q, &tmap_q, q_full, 0, kvh * G, 0, b);
-                tma_load_4d(base + sm.q + NP * 128, &tmap_q, q_full, 64, kvh * G, 0, b);
+                if (two_boxes) tma_load_4d(base + sm.q + NP * 128, &tmap_q, q_full, 64, kvh * G, 0, b);
             }
             for (int i = 0; i < first_v; ++i) {
                 if (i > 0 && i < first_k) load_k(i);
@@ -730,14 +734,16 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 tc_fence_after();
                 const uint64_t kd = kd0 + (uint64_t)(ks * (kSlot >> 4));
                 const uint32_t d = tm_s0 + sb * NP;
-                // bf16: 8 steps of 16 channels over the two 64-channel boxes; fp8: 4 steps of
-                // 32 channels against q's leading bits, then the same 4 against the rest
+                // bf16: 8 steps of 16 channels over the two 64-channel boxes (4 over the one box
+                // of head_dim 64); fp8: 4 steps of 32 channels against q's leading bits, then the
+                // same 4 against the rest
                 if (elect_one()) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         if (kFp8) mma_f8_ss(d, kd + (uint64_t)((j & 3) * 2), qd[j], idesc_qk, j > 0);
-                        else mma_f16_ss(d, kd + (uint64_t)((j >> 2) * (kBoxBytes >> 4) + (j & 3) * 2), qd[j],
-                                        idesc_qk, j > 0);
+                        else if (j < 4 || two_boxes)
+                            mma_f16_ss(d, kd + (uint64_t)((j >> 2) * (kBoxBytes >> 4) + (j & 3) * 2), qd[j],
+                                       idesc_qk, j > 0);
                     }
                     mma_commit(bar1 + 8 * hand.idx);      // s_full of tile i
                     mma_commit(k_empty(ks));
@@ -781,7 +787,9 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
                 LVSPEC_TILE_TS(tile_tr, 2, i, 2);     // V tile there
                 tc_fence_after();
                 // V^T: channels contiguous (M-major), 64-channel halves kBoxBytes apart,
-                // groups of 8 positions 1024 bytes apart.  P^T: rows contiguous in
+                // groups of 8 positions 1024 bytes apart.  (At head_dim 64 the product still
+                // has 128 rows: its upper half reads whatever follows the box in shared memory
+                // and lands in TMEM lanes nobody reads.)  P^T: rows contiguous in
                 // 16-byte chunks (N-major), chunk stride 2048, groups of 8 positions 128
                 // bytes apart.
                 const uint64_t vd = vd0 + (uint64_t)(vsl * (kSlot >> 4));
@@ -1042,7 +1050,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
                             *reinterpret_cast<uint4 *>(vrow + c * 16) = make_uint4(0, 0, 0, 0);
-                            if (!kFp8) *reinterpret_cast<uint4 *>(vrow + kBoxBytes + c * 16) = make_uint4(0, 0, 0, 0);
+                            if (two_boxes) *reinterpret_cast<uint4 *>(vrow + kBoxBytes + c * 16) = make_uint4(0, 0, 0, 0);
                         }
                     }
                 }
@@ -1166,7 +1174,7 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
                             *reinterpret_cast<uint4 *>(vrow + c * 16) = make_uint4(0, 0, 0, 0);
-                            if (!kFp8) *reinterpret_cast<uint4 *>(vrow + kBoxBytes + c * 16) = make_uint4(0, 0, 0, 0);
+                            if (two_boxes) *reinterpret_cast<uint4 *>(vrow + kBoxBytes + c * 16) = make_uint4(0, 0, 0, 0);
                         }
                     }
                 }
@@ -1224,9 +1232,9 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
                     const int n = c8 * 8 + k;
-                    if (n < M) {
+                    if (n < M && row < D) {
                         const int g = n / G, hg = n - g * G;
-                        out[(((size_t)b * gamma + g) * p.Hq + kvh * G + hg) * 128 + row] =
+                        out[(((size_t)b * gamma + g) * p.Hq + kvh * G + hg) * D + row] =
                             __float2bfloat16_rn(o8[k] * dl_s[n]);
                     }
                 }
@@ -1235,22 +1243,24 @@ attn_tc_kernel(const TcParams P, const SeqInfo seq, const __grid_constant__ CUte
             // This code runs once, on cold instruction caches, where every instruction
             // costs about ten cycles: short rolled loops, one chunk of 8 columns a turn;
             // only a last chunk that is not full takes the guarded path.
-            float *po = part_o + (size_t)c_lo * 8 * 128 + row;
+            // (TMEM lanes are channels: at head_dim 64 the upper half of the lanes holds nothing)
+            float *po = part_o + (size_t)c_lo * 8 * D + row;
+            const int m_store = row < D ? M : 0;
 #pragma unroll 1
-            for (int c8 = c_lo; c8 < c_hi; ++c8, po += 8 * 128) {
+            for (int c8 = c_lo; c8 < c_hi; ++c8, po += 8 * D) {
                 float o8[8];
                 load_acc8<kFp8>(tm_o + lane_addr, c8, o8);
                 if (kFp8) {
 #pragma unroll
                     for (int k = 0; k < 8; ++k) o8[k] *= v_scale;
                 }
-                if (c8 * 8 + 8 <= M) {
+                if (c8 * 8 + 8 <= m_store) {
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) po[k * 128] = o8[k];
+                    for (int k = 0; k < 8; ++k) po[k * D] = o8[k];
                 } else {
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
-                        if (c8 * 8 + k < M) po[k * 128] = o8[k];
+                        if (c8 * 8 + k < m_store) po[k * D] = o8[k];
                 }
             }
             if (wq == 0) {
@@ -1323,13 +1333,13 @@ EncodeTiledFn encode_fn()
 // A cache as a 4-D tensor [sequences or pages][heads][positions][128 channels] with the
 // caller's strides (in elements; the channels are contiguous).  bf16: boxes of 64 channels
 // x 128 positions; E4M3: boxes of 128 channels x 128 positions.
-bool make_kv_map(CUtensorMap *map, const void *ptr, bool fp8, int positions, int heads, int outer,
+bool make_kv_map(CUtensorMap *map, const void *ptr, bool fp8, int D, int positions, int heads, int outer,
                  int64_t s_pos, int64_t s_head, int64_t s_outer)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t esz = fp8 ? 1 : 2;
-    const cuuint64_t dims[4] = {128, (cuuint64_t)positions, (cuuint64_t)heads, (cuuint64_t)outer};
+    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)positions, (cuuint64_t)heads, (cuuint64_t)outer};
     const cuuint64_t strides[3] = {(cuuint64_t)s_pos * esz, (cuuint64_t)s_head * esz, (cuuint64_t)s_outer * esz};
     const cuuint32_t box[4] = {fp8 ? 128u : 64u, 128, 1, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -1341,12 +1351,13 @@ bool make_kv_map(CUtensorMap *map, const void *ptr, bool fp8, int positions, int
 
 // q [B][gamma][Hq][128] bf16 as a 4-D tensor; one box = 64 channels of the G heads of one
 // KV head for all gamma queries: its rows land in shared memory in the order g * G + hg
-bool make_q_map(CUtensorMap *map, const void *ptr, int B, int gamma, int Hq, int G)
+bool make_q_map(CUtensorMap *map, const void *ptr, int B, int gamma, int Hq, int G, int D)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[4] = {128, (cuuint64_t)Hq, (cuuint64_t)gamma, (cuuint64_t)B};
-    const cuuint64_t strides[3] = {256, (cuuint64_t)Hq * 256, (cuuint64_t)gamma * Hq * 256};
+    const cuuint64_t row = (cuuint64_t)D * 2;
+    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)Hq, (cuuint64_t)gamma, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {row, (cuuint64_t)Hq * row, (cuuint64_t)gamma * Hq * row};
     const cuuint32_t box[4] = {64, (cuuint32_t)G, (cuuint32_t)gamma, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(ptr), dims, strides, box,
@@ -1356,12 +1367,13 @@ bool make_q_map(CUtensorMap *map, const void *ptr, int B, int gamma, int Hq, int
 
 constexpr uint32_t kMaxSmem = 232448 - 1024;   // 227 KB less the alignment slack
 
-TcConfig pick_config(int M, int page_slots, bool fp8, bool turns)
+TcConfig pick_config(int M, int page_slots, bool fp8, bool turns, int D)
 {
     TcConfig c;
     c.n_pad = (M + 15) & ~15;
     c.page_slots = page_slots;
-    c.slot_bytes = fp8 ? kBoxBytes : kSlotBytes;
+    const bool small_tiles = fp8 || D == 64;     // one 16 KB box per tile: twice the slots
+    c.slot_bytes = small_tiles ? kBoxBytes : kSlotBytes;
     const int acc = fp8 ? 4 : 2;     // TMEM columns per padded row of O^T and the sums
     if (!turns) {
         // All groups on every tile: S^T twice.  Six ring slots when they fit, also at the
@@ -1369,8 +1381,10 @@ TcConfig pick_config(int M, int page_slots, bool fp8, bool turns)
         // flight count, and the probabilities wait in registers for the buffer anyway).
         c.sb = 2;
         const int tries[6][3] = {{3, 3, 2}, {3, 3, 1}, {2, 3, 2}, {2, 2, 2}, {2, 3, 1}, {2, 2, 1}};
+        const int tries8[6][3] = {{5, 6, 2}, {5, 5, 2}, {4, 5, 2}, {4, 4, 2}, {4, 4, 1}, {3, 3, 1}};
         for (int t = 0; t < 6; ++t) {
-            c.ks = tries[t][0]; c.vs = tries[t][1]; c.pb = tries[t][2];
+            const int *tr = small_tiles ? tries8[t] : tries[t];
+            c.ks = tr[0]; c.vs = tr[1]; c.pb = tr[2];
             if (smem_map(c).total <= kMaxSmem) break;
         }
     } else {
@@ -1383,7 +1397,7 @@ TcConfig pick_config(int M, int page_slots, bool fp8, bool turns)
         const int tries[8][3] = {{3, 3, 3}, {2, 3, 3}, {3, 2, 3}, {2, 2, 3}, {2, 2, 2}, {2, 2, 1}, {1, 2, 1}, {1, 1, 1}};
         const int tries8[8][3] = {{5, 6, 3}, {5, 5, 3}, {4, 5, 3}, {4, 4, 3}, {4, 4, 2}, {3, 3, 2}, {3, 3, 1}, {2, 2, 1}};
         for (int t = 0; t < 8; ++t) {
-            const int *tr = fp8 ? tries8[t] : tries[t];
+            const int *tr = small_tiles ? tries8[t] : tries[t];
             c.ks = tr[0]; c.vs = tr[1]; c.pb = tr[2];
             if (smem_map(c).total <= kMaxSmem) break;
         }
@@ -1408,7 +1422,7 @@ TcConfig pick_config(int M, int page_slots, bool fp8, bool turns)
 bool attn_tc_supported(const AttnParams &p)
 {
     if (p.fp8 && (p.M > kMaxRowsFp8 || p.page_size > 0 || p.branch_len != p.gamma)) return false;
-    return p.D == 128 && p.Lmax >= kTilePos && p.M <= LVSPEC_MAX_ROWS;
+    return (p.D == 128 || (p.D == 64 && !p.fp8)) && p.Lmax >= kTilePos && p.M <= LVSPEC_MAX_ROWS;
 }
 
 cudaError_t launch_attn_tc(const AttnParams &p, const SeqInfo &seq, cudaStream_t stream, int *launches)
@@ -1428,16 +1442,16 @@ cudaError_t launch_attn_tc(const AttnParams &p, const SeqInfo &seq, cudaStream_t
     bool turns = (tiles + p.n_split - 1) / p.n_split >= 96 || (fp8 && p.M <= 64);
     if (const char *e = std::getenv("LVSPEC_TC_TURNS"))
         if (e[0] == '0' || e[0] == '1') turns = e[0] == '1';
-    P.cfg = pick_config(p.M, paged ? ((tiles + p.n_split - 1) / p.n_split + 4) & ~3 : 0, fp8, turns);
+    P.cfg = pick_config(p.M, paged ? ((tiles + p.n_split - 1) / p.n_split + 4) & ~3 : 0, fp8, turns, p.D);
     if (smem_map(P.cfg).total > kMaxSmem || P.cfg.tmem_cols > 512) return cudaErrorInvalidConfiguration;
     CUtensorMap mk, mv, mq;
     const int map_len = paged ? p.page_size : p.Lmax;
     const int map_outer = paged ? p.n_pages : p.B;
-    if (!make_kv_map(&mk, p.k, fp8, map_len, p.Hkv, map_outer, p.k_sp, p.k_sh, p.k_sb) ||
-        !make_kv_map(&mv, p.v, fp8, map_len, p.Hkv, map_outer, p.v_sp, p.v_sh, p.v_sb))
+    if (!make_kv_map(&mk, p.k, fp8, p.D, map_len, p.Hkv, map_outer, p.k_sp, p.k_sh, p.k_sb) ||
+        !make_kv_map(&mv, p.v, fp8, p.D, map_len, p.Hkv, map_outer, p.v_sp, p.v_sh, p.v_sb))
         return cudaErrorInvalidValue;
     if (fp8) mq = mk;     // not used by the kernel
-    else if (!make_q_map(&mq, p.q, p.B, p.gamma, p.Hq, p.G)) return cudaErrorInvalidValue;
+    else if (!make_q_map(&mq, p.q, p.B, p.gamma, p.Hq, p.G, p.D)) return cudaErrorInvalidValue;
     const size_t smem = smem_map(P.cfg).total + 1024;
     const bool tree = p.branch_len != p.gamma;
     if ((tree && paged) || (fp8 && (tree || paged))) return cudaErrorNotSupported;

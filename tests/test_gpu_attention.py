@@ -37,8 +37,8 @@ def _case(seed, B, gamma, Hq, Hkv, D, Lmax, kv_len, span):
 
 def _skip_unless_covered(kernel, case):
     q, k = case[0], case[1]
-    if kernel == 2 and (q.shape[3] != 128 or k.shape[2] < 128):
-        pytest.skip("the tcgen05 kernel covers head_dim 128 with kv_capacity >= 128")
+    if kernel == 2 and k.shape[2] < 128:
+        pytest.skip("the tcgen05 kernel needs kv_capacity >= 128")
 
 
 def _check(ctx, oracle_mod, case, n_split=0, kernel=1):

@@ -48,6 +48,15 @@ def test_shapes(ctx, oracle_mod, organisation, shape):
     A._check(ctx, oracle_mod, A._case(31, B, gamma, Hq, Hkv, 128, Lmax, kv_len, span), n_split=n_split, kernel=2)
 
 
+@pytest.mark.parametrize("shape", [
+    (1, 4, 8, 2, 1024, [1024], [[64, 832]], 0),             # the tiny config's shape
+    (2, 8, 16, 4, 2048, [2000, 300], [[100, 1500], [0, 290]], 1),
+])
+def test_head_dim_64(ctx, oracle_mod, organisation, shape):
+    B, gamma, Hq, Hkv, Lmax, kv_len, span, n_split = shape
+    A._check(ctx, oracle_mod, A._case(36, B, gamma, Hq, Hkv, 64, Lmax, kv_len, span), n_split=n_split, kernel=2)
+
+
 @pytest.mark.parametrize("n_split", [1, 3])
 def test_scores_climbing_tile_after_tile(ctx, oracle_mod, organisation, n_split):
     """The score of every row grows by about 80 binades per 128-position tile (more than
