@@ -10,7 +10,7 @@ config's attention from one CUDA graph and prints
     prologue / dependency wait, issued their last K.Q^T and finished (%globaltimer,
     microseconds from the first stamp; first / median / last CTA), and
   * per tile of one attention CTA, clock64 stamps of the first softmax warp and of the
-    two MMA-issuing threads.
+    two MMA-issuing warps.
 
 The stamps lengthen a layer by a few tenths of a microsecond; they are for finding where
 the time goes, not for quoting a layer time (bench.py does that on the shipped library).
@@ -130,9 +130,13 @@ def main() -> None:
     if T.any():
         c0 = int(T[T > 0].min())
         print("tiles of attention CTA (split 3, KV head 2) of the last traced layer; cycles from its first stamp")
-        print("tile | K.Q^T issuer: waits for K, K there, S^T free, issued | first softmax warp (it takes every third tile): waits"
-              " for S^T, there, P buffer free, exponentials done, its turn came and m stood, P^T handed over | P.V issuer: waits"
-              " for P^T, there, V there, issued | softmax pass, per four chunks of columns: asks for S^T, has it, probabilities stored")
+        print("tile | K.Q^T issuer: waits for K, K there, S^T free, issued | first softmax warp: see below | P.V issuer: waits"
+              " for P^T, there, V there, issued | softmax pass of that warp, per four chunks of columns (tiles in turn"
+              " only): asks for S^T, has it, probabilities stored")
+        print("first softmax warp, all groups on every tile (short streams per CTA, bf16 cache): waits for S^T, there,"
+              " exponentials done, group agreed on the guard, P buffer free, P^T handed over")
+        print("first softmax warp, groups take the tiles in turn (it has every third tile; long streams, fp8 cache): waits"
+              " for S^T, there, P buffer free, exponentials done, its turn came and m stood, P^T handed over")
         rel = lambda a: " ".join(f"{int(x) - c0:6d}" if x else "     -" for x in a)
         for i in range(32):
             if not T[:, i].any():
