@@ -78,7 +78,7 @@ typedef struct {
 
 #define LVSPEC_KERNEL_DEFAULT 0
 #define LVSPEC_KERNEL_SIMT    1 /* plain CUDA-core kernel: any supported shape */
-#define LVSPEC_KERNEL_TCGEN05 2 /* TMA + tcgen05 tensor-core kernel */
+#define LVSPEC_KERNEL_TCGEN05 2 /* TMA + tcgen05 tensor-core kernel: kv_capacity >= 128 (the default then) */
 
 /* Parameters of the rule.  n_loose >= 0 gives the number of loosened positions
  * directly; n_loose < 0 derives it from lambda as floor(lambda * gamma + 1e-9)
