@@ -325,8 +325,12 @@ lvspec_status_t lvspec_verify_attention_paged(lvspec_ctx_t *ctx, const lvspec_at
  * Arithmetic: the 8-bit tiles go to the tensor cores as they are; q and the
  * probabilities are each split into two E4M3 terms (leading four significant bits and
  * the rest) so that they lose no more than they would as bf16; accumulation is fp32.
- * Probabilities of a row are held within 2^8 above and about 2^11 below those of the
- * largest score seen so far; terms smaller than that by another factor of 2^6 vanish.
+ * Range: E4M3 has 17 binades.  A row's reference is set so that the largest score of the
+ * split's first tile has probability 2^3, and moves up (with a rescale of the
+ * accumulators) when a later score exceeds that by more than 2^5.  A probability keeps
+ * eight significant bits down to 2^5 below the first tile's largest, four bits down to
+ * 2^9 below, and vanishes 2^12 below it: a row that holds most of its mass that far (8
+ * nats) under its largest score is beyond this call; the bf16 call has no such limit.
  * Tolerances against the plain definition on the decoded cache: those of the bf16 call.
  * UNSUPPORTED for head_dim other than 128, for LVSPEC_KERNEL_SIMT, for more than 80
  * query rows per KV head (gamma * Hq / Hkv), and for kv_capacity < 128. */
