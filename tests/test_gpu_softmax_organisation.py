@@ -144,3 +144,22 @@ def test_random_shapes_with_moving_references(ctx, oracle_mod, organisation):
         assert np.isfinite(out).all() and np.isfinite(mass).all(), case_id
         assert (np.abs(out - ref_out) <= 1e-2 + 1e-2 * np.abs(ref_out)).all(), case_id
         assert np.abs(mass - ref_mass).max() <= 2.0 ** -9, (case_id, np.abs(mass - ref_mass).max())
+
+
+@pytest.mark.parametrize("ring", ["2,2,1,2", "2,2,2,2", "3,2,2,3", "1,1,1,2", "2,3,3,3"])
+def test_turns_with_fewer_buffers(ctx, oracle_mod, monkeypatch, ring):
+    """LVSPEC_TC_RING="K slots,V slots,P buffers,S buffers" (read at every launch) forces the
+    buffer counts that large row counts make the library fall back to: groups that share
+    P^T and S^T buffers wait for tiles other groups hold, and the hand-over barriers, indexed
+    by tile, must still tell every phase apart.  One CTA streams 32 tiles, with moving
+    reference exponents in the second case."""
+    monkeypatch.setenv("LVSPEC_TC_TURNS", "1")
+    monkeypatch.setenv("LVSPEC_TC_RING", ring)
+    A._check(ctx, oracle_mod, A._case(37, 1, 8, 40, 8, 128, 4096, [4001], [[256, 3000]]), n_split=1, kernel=2)
+    q, k, v, kv_len, span = A._case(38, 2, 4, 8, 2, 128, 2304, [2304, 700], [[100, 2000], [0, 650]])
+    k = W.f32_to_bf16_bits(W.bf16_bits_to_f32(k) * 6.0)
+    from gpu_util import run_attention
+    ref_out, ref_mass = oracle_mod.verify_attention(q, k, v, kv_len, span)
+    out, mass = run_attention(ctx, q, k, v, kv_len, span, n_split=2, kernel=2)
+    assert (np.abs(out - ref_out) <= 1e-2 + 1e-2 * np.abs(ref_out)).all()
+    assert np.abs(mass - ref_mass).max() <= 2.0 ** -9
