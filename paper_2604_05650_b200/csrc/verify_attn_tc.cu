@@ -1,4 +1,4 @@
-// Verification attention with fused visual mass: TMA + tcgen05 kernel (D = 128).
+// Verification attention with fused visual mass: TMA + tcgen05 kernel (D = 128 or 64).
 //
 // One CTA owns one KV split of one (sequence, KV head) and the M = gamma * G
 // query rows that read this head.  The GQA-grouped queries are the small side
@@ -48,10 +48,14 @@
 // 2 x 128 channels); a probability is split by the softmax threads, head and rest sit
 // in neighbouring columns of P^T, and V^T.P^T and the sum products run with N = 2 x
 // rows: accumulator column 2n holds the head's part of row n, column 2n + 1 the rest's,
-// added once in the epilogue.  Probabilities are kept within E4M3's range by holding
-// the reference exponent at most 8 binades below the largest score seen (the first
-// position sits at 2^4).  The K scale folds into the softmax scale, the V scale into the
-// epilogue.
+// added once in the epilogue.  Probabilities are kept within E4M3's range by the
+// reference exponent: the largest score of the split's first tile gets probability 2^3,
+// and a later score that would pass 2^8 moves the reference up.  The K scale folds into the
+// softmax scale, the V scale into the epilogue.
+//
+// head_dim 64: one 64-channel box per K or V tile and four K.Q^T steps; the P.V product
+// keeps its 128 rows, of which the upper 64 read what follows the box in shared memory
+// and fill TMEM lanes nobody reads.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
