@@ -714,7 +714,7 @@ def time_fp8_attention(cfg, ctx, stream, ks, vs_, qs, torch, dev, peak):
     nbytes = cfg.kv_bytes_per_layer // 2 + 2 * B * Hkv * 4 + 2 * B * g * Hq * D * 2 + B * g * Hq * 4
     gbs = nbytes / (us * 1e-6) / 1e9
     return {"us_per_layer": us, "layers_in_graph": n_layers, "bytes_per_layer": nbytes, "achieved_gbs": gbs,
-            "frac_of_peak": gbs / peak, "splits": ctx.attention_splits(shape, L), "cache": "E4M3, one scale per KV head"}
+            "frac_of_peak": gbs / peak, "splits": ctx.attention_splits(shape, L, fp8=True), "cache": "E4M3, one scale per KV head"}
 
 
 def time_paged_attention(cfg, ctx, stream, ks, vs_, qs, torch, dev, peak):

@@ -132,6 +132,9 @@ uint64_t lvspec_launch_count(const lvspec_ctx_t *ctx);
  * `max_kv_len` (what n_split = 0 resolves to); 0 on invalid input. */
 int32_t lvspec_attention_splits(const lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
                                 int32_t max_kv_len);
+/* The same for lvspec_verify_attention_fp8 (half the bytes per tile: it takes more splits). */
+int32_t lvspec_attention_splits_fp8(const lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                    int32_t max_kv_len);
 
 /* Scratch memory.  A context owns one scratch buffer on its device (split
  * partials of the attention, argmax partials of the acceptance pass, cosines of

@@ -26,7 +26,7 @@ MAX_BATCH, MAX_ROWS, MAX_GAMMA = 128, 128, 64
 EXPORTS = (
     "lvspec_create", "lvspec_destroy", "lvspec_set_stream", "lvspec_device_status",
     "lvspec_last_error", "lvspec_status_string", "lvspec_launch_count",
-    "lvspec_attention_splits", "lvspec_verify_attention", "lvspec_verify_attention_host",
+    "lvspec_attention_splits", "lvspec_attention_splits_fp8", "lvspec_verify_attention", "lvspec_verify_attention_host",
     "lvspec_loose_accept", "lvspec_loose_accept_ex", "lvspec_loose_accept_host",
     "lvspec_loose_accept_static", "lvspec_row_inv_norms", "lvspec_visual_relevance",
     "lvspec_selftest_wait_expiry", "lvspec_loose_accept_emit",
@@ -98,6 +98,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lvspec_launch_count.restype = u64
     lib.lvspec_attention_splits.argtypes = [vp, S, i32]
     lib.lvspec_attention_splits.restype = i32
+    lib.lvspec_attention_splits_fp8.argtypes = [vp, S, i32]
+    lib.lvspec_attention_splits_fp8.restype = i32
     lib.lvspec_verify_attention.argtypes = [vp, S, vp, vp, vp, vp, vp, vp, vp]
     lib.lvspec_verify_attention_host.argtypes = [vp, S, vp, vp, vp, vp, vp, vp, vp]
     lib.lvspec_verify_attention_fp8.argtypes = [vp, S, vp, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -118,7 +120,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
                                                ctypes.c_char_p, ctypes.c_size_t]
     for name in EXPORTS:
         fn = getattr(lib, name)
-        if fn.restype is ctypes.c_int and name not in ("lvspec_attention_splits",):
+        if fn.restype is ctypes.c_int and name not in ("lvspec_attention_splits", "lvspec_attention_splits_fp8"):
             fn.restype = ctypes.c_int
     if path == LIB_PATH:
         _lib = lib
@@ -207,8 +209,9 @@ class Context:
     def launch_count(self) -> int:
         return int(self._lib.lvspec_launch_count(self._h))
 
-    def attention_splits(self, shape: AttnShape, max_kv_len: int) -> int:
-        return int(self._lib.lvspec_attention_splits(self._h, ctypes.byref(shape), int(max_kv_len)))
+    def attention_splits(self, shape: AttnShape, max_kv_len: int, fp8: bool = False) -> int:
+        fn = self._lib.lvspec_attention_splits_fp8 if fp8 else self._lib.lvspec_attention_splits
+        return int(fn(self._h, ctypes.byref(shape), int(max_kv_len)))
 
     # -- lvspec_verify_attention ------------------------------------------------
     def verify_attention(self, shape: AttnShape, q, k_cache, v_cache, kv_len, visual_span,

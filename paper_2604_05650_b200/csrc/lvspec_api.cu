@@ -531,6 +531,13 @@ int32_t lvspec_attention_splits(const lvspec_ctx_t *ctx, const lvspec_attn_shape
     return shape->n_split > 0 ? shape->n_split : choose_splits(ctx, shape, max_kv_len);
 }
 
+int32_t lvspec_attention_splits_fp8(const lvspec_ctx_t *ctx, const lvspec_attn_shape_t *shape,
+                                    int32_t max_kv_len)
+{
+    if (!ctx || !shape || shape->batch < 1 || shape->n_kv_heads < 1 || max_kv_len < 1) return 0;
+    return shape->n_split > 0 ? shape->n_split : choose_splits(ctx, shape, max_kv_len, true);
+}
+
 lvspec_status_t lvspec_last_device_status(lvspec_ctx_t *ctx, uint32_t *flags)
 {
     return lvspec_device_status(ctx, flags);
